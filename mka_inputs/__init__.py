@@ -1,0 +1,8 @@
+"""Seeded synthetic inputs for the FastMKA hot path.
+
+This package holds only the input recipe: a counter-based pseudo-random
+generator and the tensor shapes of the benchmark configurations.  It contains
+none of the attention / routing arithmetic, and it is the one module that both
+the CPU oracle's tests and the CUDA path's tests and benchmark may import.
+"""
+from .generator import approx_normal, CONFIGS, WorkloadConfig, make_tensor, TENSOR_IDS  # noqa: F401

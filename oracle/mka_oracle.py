@@ -1,0 +1,234 @@
+"""numpy front end of the CPU oracle (``mka_oracle.c``) -- TEST INFRASTRUCTURE ONLY.
+
+Nothing in the product package may import this module; it exists so that the
+tests, the smoke check and the benchmark's cpu-baseline leg can evaluate the
+paper's definitions (Eq. 5, Alg. 1, the router, the derived backward) in fp64.
+
+The wrappers only marshal arrays: they loop over (batch, head), hand one head
+problem at a time to the C routines, and sum the per-head router-logit
+gradients over heads (the gate is one per token, shared by all heads).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mka_oracle.c")
+_LIB = os.path.join(_HERE, "libmka_oracle.so")
+_lib = None
+
+ROUTE_SOFT, ROUTE_UNIFORM, ROUTE_TOP1, ROUTE_TOP2 = 0, 1, 2, 3
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP) if the library is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.orc_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().orc_num_threads())
+
+
+_DP = ctypes.POINTER(ctypes.c_double)
+_LP = ctypes.POINTER(ctypes.c_int64)
+
+
+def _p(a: Optional[np.ndarray]):
+    if a is None:
+        return ctypes.cast(None, _DP)
+    assert a.dtype == np.float64 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(_DP)
+
+
+def _f64(a) -> np.ndarray:
+    if hasattr(a, "detach"):  # torch tensor
+        a = a.detach().to("cpu").double().numpy()
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def visible(level: int, p: int, W: int, n: int, decode: bool = False):
+    lo, hi = ctypes.c_int64(), ctypes.c_int64()
+    _load().orc_visible(ctypes.c_int(level), ctypes.c_int64(p), ctypes.c_int64(W), ctypes.c_int64(n),
+                        ctypes.c_int(int(decode)), ctypes.byref(lo), ctypes.byref(hi))
+    return lo.value, hi.value
+
+
+def router(R, W_r, b_r=None, route: int = ROUTE_SOFT):
+    """R[..., D], W_r[D, 3], b_r[3] -> gate[..., 3] (fp64), idx[..., 2] (int8)."""
+    R = _f64(R)
+    lead = R.shape[:-1]
+    D = R.shape[-1]
+    R2 = R.reshape(-1, D)
+    W_r = _f64(W_r)
+    assert W_r.shape == (D, 3)
+    b = None if b_r is None else _f64(b_r)
+    gate = np.empty((R2.shape[0], 3), np.float64)
+    idx = np.empty((R2.shape[0], 2), np.int8)
+    rc = _load().orc_router(_p(R2), _p(W_r), _p(b), ctypes.c_int64(R2.shape[0]), ctypes.c_int64(D),
+                            ctypes.c_int(route), _p(gate), idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int8)))
+    assert rc == 0
+    return gate.reshape(*lead, 3), idx.reshape(*lead, 2)
+
+
+def _head_args(Qh, Ks, Vs, gate_b, W, q_off, tau, decode):
+    T, d = Qh.shape
+    args = [_p(Qh), ctypes.c_int64(T), ctypes.c_int64(d)]
+    for l in range(3):
+        n = Ks[l].shape[0]
+        args += [_p(Ks[l]) if n else ctypes.cast(None, _DP), _p(Vs[l]) if n else ctypes.cast(None, _DP),
+                 ctypes.c_int64(n)]
+    args += [_p(gate_b), ctypes.c_int64(W), ctypes.c_int64(q_off), ctypes.c_double(tau), ctypes.c_int(int(decode))]
+    return args
+
+
+def _prep(Q, K, V, gate):
+    Q = _f64(Q)
+    K = [_f64(k) for k in K]
+    V = [_f64(v) for v in V]
+    gate = _f64(gate)
+    B, H, T, d = Q.shape
+    assert gate.shape == (B, T, 3)
+    for l in range(3):
+        assert K[l].shape == V[l].shape and K[l].shape[:2] == (B, H) and K[l].shape[3] == d
+    return Q, K, V, gate, B, H, T, d
+
+
+def _rows_arg(rows, T):
+    if rows is None:
+        return None, ctypes.cast(None, _LP), T
+    r = np.ascontiguousarray(rows, dtype=np.int64)
+    assert r.ndim == 1 and (r >= 0).all() and (r < T).all()
+    return r, r.ctypes.data_as(_LP), r.shape[0]
+
+
+def fwd(Q, K: Sequence, V: Sequence, gate, window: int, q_offset: int = 0, scale: Optional[float] = None,
+        mode: str = "fast", decode: bool = False, rows=None, heads=None):
+    """Forward of the operator.
+
+    Q[B,H,T,d]; K[l], V[l] : [B,H,N_l,d]; gate[B,T,3].  mode "fast" = Eq. 5, "full" = Alg. 1.
+    rows: optional 1-D list of query indices evaluated for every head (output then has
+    len(rows) rows).  heads: optional list of (b, h) pairs; other heads are left as NaN.
+    Returns O[B,H,R,d] and LSE[B,H,R] (LSE is None in "full" mode).
+    """
+    Q, K, V, gate, B, H, T, d = _prep(Q, K, V, gate)
+    tau = (1.0 / np.sqrt(d)) if scale is None or scale <= 0 else float(scale)
+    rkeep, rptr, R = _rows_arg(rows, T)
+    O = np.full((B, H, R, d), np.nan)
+    LSE = np.full((B, H, R), np.nan)
+    lib = _load()
+    pairs = heads if heads is not None else [(b, h) for b in range(B) for h in range(H)]
+    for b, h in pairs:
+        Ks = [np.ascontiguousarray(K[l][b, h]) for l in range(3)]
+        Vs = [np.ascontiguousarray(V[l][b, h]) for l in range(3)]
+        Qh = np.ascontiguousarray(Q[b, h])
+        gb = np.ascontiguousarray(gate[b])
+        o = np.empty((R, d))
+        args = _head_args(Qh, Ks, Vs, gb, window, q_offset, tau, decode) + [rptr, ctypes.c_int64(R), _p(o)]
+        if mode == "fast":
+            ls = np.empty((R,))
+            rc = lib.orc_fwd_fast_head(*args, _p(ls))
+            LSE[b, h] = ls
+        elif mode == "full":
+            rc = lib.orc_fwd_full_head(*args)
+        else:
+            raise ValueError(mode)
+        assert rc == 0
+        O[b, h] = o
+    return O, (LSE if mode == "fast" else None)
+
+
+def fwd_recursive(Q, K, V, gate, window: int, q_offset: int = 0, scale: Optional[float] = None,
+                  block: int = 128, decode: bool = False):
+    """Eq. 6-8 / Eq. 11-14 evaluated level by level in key blocks (checks Theorem 1)."""
+    Q, K, V, gate, B, H, T, d = _prep(Q, K, V, gate)
+    tau = (1.0 / np.sqrt(d)) if scale is None or scale <= 0 else float(scale)
+    O = np.empty((B, H, T, d))
+    LSE = np.empty((B, H, T))
+    lib = _load()
+    for b in range(B):
+        for h in range(H):
+            Ks = [np.ascontiguousarray(K[l][b, h]) for l in range(3)]
+            Vs = [np.ascontiguousarray(V[l][b, h]) for l in range(3)]
+            o = np.empty((T, d))
+            ls = np.empty((T,))
+            rc = lib.orc_fwd_recursive_head(*_head_args(np.ascontiguousarray(Q[b, h]), Ks, Vs,
+                                                        np.ascontiguousarray(gate[b]), window, q_offset, tau, decode),
+                                            ctypes.c_int64(block), _p(o), _p(ls))
+            assert rc == 0
+            O[b, h], LSE[b, h] = o, ls
+    return O, LSE
+
+
+def bwd(Q, K, V, gate, dO, window: int, q_offset: int = 0, scale: Optional[float] = None,
+        decode: bool = False, rows=None, heads=None, want_kv: bool = True):
+    """Gradients of <dO, O> for the "fast" operator.
+
+    Returns dict with dQ[B,H,R,d], dK[l], dV[l] ([B,H,N_l,d]; complete only when rows is
+    None), G[B,H,R,3] (per-head router-logit gradient) and dG[B,R,3] = sum over heads.
+    With `heads`, only those (b, h) pairs are evaluated (others NaN; dG then sums only them).
+    """
+    Q, K, V, gate, B, H, T, d = _prep(Q, K, V, gate)
+    dO = _f64(dO)
+    assert dO.shape == Q.shape
+    tau = (1.0 / np.sqrt(d)) if scale is None or scale <= 0 else float(scale)
+    rkeep, rptr, R = _rows_arg(rows, T)
+    dQ = np.full((B, H, R, d), np.nan)
+    G = np.full((B, H, R, 3), np.nan)
+    dK = [np.full(K[l].shape, np.nan) for l in range(3)] if want_kv else None
+    dV = [np.full(V[l].shape, np.nan) for l in range(3)] if want_kv else None
+    lib = _load()
+    pairs = heads if heads is not None else [(b, h) for b in range(B) for h in range(H)]
+    null = ctypes.cast(None, _DP)
+    for b, h in pairs:
+        Ks = [np.ascontiguousarray(K[l][b, h]) for l in range(3)]
+        Vs = [np.ascontiguousarray(V[l][b, h]) for l in range(3)]
+        dq = np.empty((R, d))
+        g = np.empty((R, 3))
+        outs = []
+        bufs = []
+        for l in range(3):
+            if want_kv:
+                a, c = np.empty(Ks[l].shape), np.empty(Vs[l].shape)
+                bufs.append((a, c))
+                outs += [_p(a), _p(c)]
+            else:
+                outs += [null, null]
+        rc = lib.orc_bwd_head(*_head_args(np.ascontiguousarray(Q[b, h]), Ks, Vs, np.ascontiguousarray(gate[b]),
+                                          window, q_offset, tau, decode),
+                              _p(np.ascontiguousarray(dO[b, h])), rptr, ctypes.c_int64(R), _p(dq), *outs, _p(g))
+        assert rc == 0
+        dQ[b, h], G[b, h] = dq, g
+        if want_kv:
+            for l in range(3):
+                dK[l][b, h], dV[l][b, h] = bufs[l]
+    dG = np.zeros((B, R, 3))
+    for b, h in pairs:
+        dG[b] += G[b, h]
+    return {"dQ": dQ, "dK": dK, "dV": dV, "G": G, "dG": dG}
+
+
+def router_bwd(R, dG):
+    """dW_r[D,3] = sum over tokens of R^T dG, db_r[3] = sum dG (soft routing; the gate's
+    softmax Jacobian is already folded into dG)."""
+    R = _f64(R)
+    dG = _f64(dG)
+    D = R.shape[-1]
+    dW = R.reshape(-1, D).T @ dG.reshape(-1, 3)
+    return dW, dG.reshape(-1, 3).sum(0)
