@@ -1,0 +1,187 @@
+/*
+ * mka.h -- C ABI of the B200 (sm_100a) FastMKA attention library.
+ *
+ * The operator (paper, "Theoretical Formulation", Eq. 5): for every query token t a router gate
+ * lambda_t in R^3 (non-negative, sums to one) weighs three memory levels -- L1 local window,
+ * L2 session memory, L3 long-term slots -- and the output is the gated mixture of
+ * exponentiated scores under ONE normalisation:
+ *
+ *     O_t = sum_l lambda_{t,l} sum_{j in vis_l(t)} exp(s_{t,l,j}) v_{l,j}  /  Z_t
+ *     Z_t = sum_l lambda_{t,l} sum_{j in vis_l(t)} exp(s_{t,l,j}),   s_{t,l,j} = scale * q_t . k_{l,j}
+ *
+ * evaluated block-wise with a running maximum (Eq. 11-14; block partition Eq. 2-4, Alg. 3).
+ * Visibility: with p = t + q_offset the position of query t on the key timeline,
+ *     L1: j in (p - window, p]      (a causal window that ends at, and includes, the query's own row)
+ *     L2: j in [0, p]               (causal prefix; one session entry per token)
+ *     L3: j in [0, n_3)             (every recalled slot)
+ * each intersected with [0, n_l).  A level with n_l = 0, or a row whose gate for that level is 0,
+ * contributes nothing (Local-MKA = levels 1,2 only; "L1 only" = standard attention).
+ *
+ * General rules for every entry point
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  Structs (mka_shape,
+ *     mka_level[3], ...) are read on the host during the call.
+ *   - The caller owns every buffer; the library allocates no device memory and keeps no state
+ *     between calls.  Scratch memory comes from the caller as `ws` (size from mka_workspace_bytes).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls only enqueue work;
+ *     they do not synchronise.  Outputs are fully overwritten.
+ *   - Errors are reported by return code only; arguments are validated on the host before anything
+ *     is launched, and nothing is launched when validation fails.  No entry point aborts or traps.
+ *   - Head width d must be 32, 64, 96 or 128 (decode and the tensor-core forward: 64 or 128).  bf16 tensors
+ *     need 16-byte aligned base pointers and strides that are multiples of 8 elements.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point returns MKA_ERR_CUDA.
+ */
+#ifndef MKA_H_
+#define MKA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MKA_OK = 0,
+    MKA_ERR_ARG = 1,          /* null pointer, bad enum value */
+    MKA_ERR_SHAPE = 2,        /* non-positive size, unsupported head width, window < 1 */
+    MKA_ERR_ALIGN = 3,        /* pointer or stride alignment */
+    MKA_ERR_WORKSPACE = 4,    /* ws == NULL or ws_bytes too small */
+    MKA_ERR_UNSUPPORTED = 5,  /* combination not implemented (e.g. MKA_MODE_FULL backward) */
+    MKA_ERR_CUDA = 6,         /* a CUDA runtime call failed (no device, launch failure) */
+    MKA_ERR_TIMEOUT = 7       /* a bounded device-side wait expired (see mka_device_status) */
+} mka_status;
+
+typedef enum { MKA_BF16 = 0, MKA_F32 = 1 } mka_dtype;
+
+/* MKA_MODE_FAST: Eq. 5 (FastMKA: one attention pass, one normalisation).
+ * MKA_MODE_FULL: Alg. 1 (Symbolic MKA): one softmax attention per level, outputs mixed by the gate. */
+typedef enum { MKA_MODE_FAST = 0, MKA_MODE_FULL = 1 } mka_mode;
+
+/* Routing variants of the gate (Alg. 1 "lambda <- softmax(MLP(q))"; hard top-k and fixed 1/3 are the
+ * routing-ablation variants of Table 10). */
+typedef enum { MKA_ROUTE_SOFT = 0, MKA_ROUTE_UNIFORM = 1, MKA_ROUTE_TOP1 = 2, MKA_ROUTE_TOP2 = 3 } mka_route;
+
+/* mka_shape.flags */
+#define MKA_FLAG_FORCE_SIMT 1u   /* run the CUDA-core kernels even where a tensor-core kernel exists */
+
+/* which = argument of mka_workspace_bytes */
+#define MKA_WS_FWD 0
+#define MKA_WS_DECODE 1
+#define MKA_WS_BWD 2
+
+/* One memory level's key/value source: k, v are [B, H, n, d] with d contiguous and explicit strides
+ * (in ELEMENTS) for the batch, head and row dimensions.  n may be 0 (then k, v may be NULL). */
+typedef struct mka_level {
+    const void *k, *v;
+    int64_t n;
+    int64_t stride_b, stride_h, stride_n;
+} mka_level;
+
+/* Gradient destinations for one level, same geometry as mka_level. */
+typedef struct mka_level_grad {
+    void *dk, *dv;
+    int64_t n;
+    int64_t stride_b, stride_h, stride_n;
+} mka_level_grad;
+
+/* Problem shape in the paper's notation: B batch, H heads, T query tokens, d head width, D model
+ * width (router input width); window = W of the L1 level; q_offset = key-timeline position of query 0;
+ * scale = tau of Eq. 3 (<= 0 selects 1/sqrt(d)). */
+typedef struct mka_shape {
+    int32_t B, H, T, d, D;
+    int32_t window;
+    int32_t q_offset;
+    float scale;
+    int32_t dtype;   /* mka_dtype of Q, K, V, O, dO, dQ, dK, dV */
+    int32_t mode;    /* mka_mode */
+    uint32_t flags;  /* MKA_FLAG_* */
+} mka_shape;
+
+/* Split table of the decode kernel: level l is cut into n_chunks[l] chunks of chunk_rows rows (the last
+ * one shorter); chunk c of level l covers rows [c*chunk_rows, min(n_l, (c+1)*chunk_rows)). */
+typedef struct mka_decode_plan_t {
+    int64_t chunk_rows;
+    int64_t n_chunks[3];
+    int64_t total_chunks;   /* per (batch, head) */
+} mka_decode_plan_t;
+
+/* Key-tile range of one 128-row query tile on one level, in units of 128-row key tiles:
+ * tiles [first, end) hold at least one visible pair; tiles [full_first, full_end) within it are
+ * visible to every row of the query tile and need no element mask. */
+typedef struct mka_tile_range {
+    int64_t first, end, full_first, full_end;
+} mka_tile_range;
+
+const char* mka_status_str(mka_status s);
+
+/*
+ * Router gate (Alg. 1 step 12 / Alg. 2 step 5, read as one linear layer followed by a softmax over
+ * the three levels; one gate per token, shared by all heads).
+ *   R        [rows, D] router input, row-major, r_dtype (bf16 or f32)
+ *   W_r      [D, 3] f32, b_r [3] f32 or NULL (zero bias)
+ *   route    MKA_ROUTE_*: SOFT = softmax; UNIFORM = 1/3 each; TOP1/TOP2 = keep the 1/2 largest logits
+ *            (ties go to the lower level index), renormalise the kept gates, others exactly 0
+ *   gate     [rows, 3] f32 out
+ *   log2_gate[rows, 3] f32 out or NULL: log2 of the gate (-inf where the gate is 0)
+ *   route_idx[rows, 2] int8 out or NULL: kept level indices ascending, -1 = unused slot
+ *            (both -1 for SOFT and UNIFORM)
+ * rows == 0 is valid and launches nothing.
+ */
+mka_status mka_router(const void* R, const float* W_r, const float* b_r, int64_t rows, int32_t D,
+                      int32_t r_dtype, int32_t route, float* gate, float* log2_gate, int8_t* route_idx,
+                      void* stream);
+
+/* Bytes of caller-provided scratch the given entry point needs (host function, no CUDA call).
+ * n_level = rows of the three levels.  Returns 0 on invalid arguments. */
+size_t mka_workspace_bytes(const mka_shape* shape, const int64_t n_level[3], int32_t which);
+
+/*
+ * Fused forward (Eq. 5 block-wise with the running maximum of Eq. 11-14; MKA_MODE_FULL: Alg. 1).
+ *   Q    [B, H, T, d] contiguous;  L[3] level sources;  gate [B, T, 3] f32 (an INPUT: >= 0)
+ *   O    [B, H, T, d] out, same dtype as Q (rounded once, to nearest even, for bf16)
+ *   LSE  [B, H, T] f32 out or NULL: natural log of Z_t (-inf and O = 0 where nothing is visible);
+ *        not written in MKA_MODE_FULL
+ * bf16 with d in {64,128} runs the TMA + tcgen05 kernel; f32, MKA_MODE_FULL and MKA_FLAG_FORCE_SIMT
+ * run the CUDA-core kernel.
+ */
+mka_status mka_fwd(const mka_shape* shape, const void* Q, const mka_level L[3], const float* gate,
+                   void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Split-KV single-token decode: Eq. 5 for T == 1 where EVERY cached row of every level is visible
+ * (window and q_offset are ignored).  Each chunk of the split table produces an un-gated partial
+ * (max, sum, accumulator); a second kernel combines them with the gate in log-sum-exp form.
+ *   q [B, H, d];  gate [B, 3] f32;  O [B, H, d];  LSE [B, H] f32 or NULL.
+ */
+mka_status mka_decode(const mka_shape* shape, const void* q, const mka_level L[3], const float* gate,
+                      void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Backward of mka_fwd in MKA_MODE_FAST (derived from Eq. 5; the paper prints no backward).  With
+ * p = lambda exp(s - LSE) on the visible set and D_t = dO_t . O_t:
+ *   dV = p^T dO,  dS = p (dO v^T - D),  dQ = scale dS K,  dK = scale dS^T Q,
+ *   dG[b,t,l] = sum over heads and visible j of dS   (gradient w.r.t. the router LOGIT of level l),
+ *   dW_r = R^T dG,  db_r = sum dG.
+ *   O, LSE: outputs of mka_fwd;  dO [B,H,T,d];  R [B*T, D] router input in r_dtype (NULL skips dW_r, db_r)
+ *   dQ [B,H,T,d];  dL[3] gradient destinations (a level with n == 0 is skipped);  dG [B,T,3] f32;
+ *   dW_r [D,3] f32 or NULL;  db_r [3] f32 or NULL.
+ */
+mka_status mka_bwd(const mka_shape* shape, const void* Q, const mka_level L[3], const float* gate,
+                   const void* O, const float* LSE, const void* dO, const void* R, int32_t r_dtype,
+                   void* dQ, const mka_level_grad dL[3], float* dG, float* dW_r, float* db_r,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/* Integer bookkeeping, exposed so that it can be checked bit for bit (host functions, no CUDA call). */
+mka_status mka_decode_plan(const int64_t n_level[3], int32_t B, int32_t H, int32_t d, mka_decode_plan_t* plan);
+mka_status mka_fwd_tile_range(const mka_shape* shape, const int64_t n_level[3], int32_t level,
+                              int64_t q_tile, mka_tile_range* out);
+
+/* Synchronises `stream` and returns the device status word that the kernels of the last call using
+ * `ws` left there: MKA_OK, or MKA_ERR_TIMEOUT when a bounded wait inside a kernel gave up (the
+ * kernel then released its resources and returned; outputs of that call are invalid). */
+mka_status mka_device_status(const void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MKA_H_ */

@@ -1,0 +1,237 @@
+"""Thin ctypes binding of the C-ABI library (``libmka_b200.so``): argument marshalling only.
+
+Function names match ``include/mka.h``.  Tensors are ``torch`` CUDA tensors used purely as device
+memory; every step of the path runs inside the library's kernels.  There is no fallback: if the
+library has not been built the import fails, and every call raises ``MkaError`` on a non-zero status.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmka_b200.so")
+
+MKA_BF16, MKA_F32 = 0, 1
+MKA_MODE_FAST, MKA_MODE_FULL = 0, 1
+MKA_ROUTE_SOFT, MKA_ROUTE_UNIFORM, MKA_ROUTE_TOP1, MKA_ROUTE_TOP2 = 0, 1, 2, 3
+MKA_FLAG_FORCE_SIMT = 1
+MKA_WS_FWD, MKA_WS_DECODE, MKA_WS_BWD = 0, 1, 2
+TILE = 128
+
+EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
+           "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status"]
+
+
+class MkaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: status {code} ({status_str(code)})")
+
+
+class mka_level(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("n", ctypes.c_int64),
+                ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64)]
+
+
+class mka_level_grad(ctypes.Structure):
+    _fields_ = [("dk", ctypes.c_void_p), ("dv", ctypes.c_void_p), ("n", ctypes.c_int64),
+                ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64)]
+
+
+class mka_shape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("D", ctypes.c_int32), ("window", ctypes.c_int32), ("q_offset", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32),
+                ("flags", ctypes.c_uint32)]
+
+
+class mka_decode_plan_t(ctypes.Structure):
+    _fields_ = [("chunk_rows", ctypes.c_int64), ("n_chunks", ctypes.c_int64 * 3), ("total_chunks", ctypes.c_int64)]
+
+
+class mka_tile_range(ctypes.Structure):
+    _fields_ = [("first", ctypes.c_int64), ("end", ctypes.c_int64), ("full_first", ctypes.c_int64),
+                ("full_end", ctypes.c_int64)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_20586_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    lib.mka_status_str.restype = ctypes.c_char_p
+    lib.mka_status_str.argtypes = [ctypes.c_int]
+    lib.mka_workspace_bytes.restype = ctypes.c_size_t
+    lib.mka_workspace_bytes.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32]
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    lib.mka_router.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+    lib.mka_fwd.argtypes = [ctypes.POINTER(mka_shape), vp, ctypes.POINTER(mka_level), vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.mka_decode.argtypes = lib.mka_fwd.argtypes
+    lib.mka_bwd.argtypes = [ctypes.POINTER(mka_shape), vp, ctypes.POINTER(mka_level), vp, vp, vp, vp, vp, i32, vp,
+                            ctypes.POINTER(mka_level_grad), vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.mka_decode_plan.argtypes = [ctypes.POINTER(ctypes.c_int64), i32, i32, i32, ctypes.POINTER(mka_decode_plan_t)]
+    lib.mka_fwd_tile_range.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(ctypes.c_int64), i32, i64,
+                                       ctypes.POINTER(mka_tile_range)]
+    lib.mka_device_status.argtypes = [vp, vp]
+    for name in EXPORTS:
+        if name not in ("mka_status_str", "mka_workspace_bytes"):
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+lib = _load()
+
+
+def status_str(code: int) -> str:
+    return lib.mka_status_str(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise MkaError(code, where)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return MKA_BF16
+    if t.dtype == torch.float32:
+        return MKA_F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _n_level(n) -> ctypes.Array:
+    return (ctypes.c_int64 * 3)(*[int(x) for x in n])
+
+
+def make_shape(B, H, T, d, D=0, window=1, q_offset=0, scale=0.0, dtype=MKA_BF16, mode=MKA_MODE_FAST, flags=0) -> mka_shape:
+    return mka_shape(B, H, T, d, D, window, q_offset, scale, dtype, mode, flags)
+
+
+def _levels(K: Sequence[Optional[torch.Tensor]], V: Sequence[Optional[torch.Tensor]]):
+    arr = (mka_level * 3)()
+    for l in range(3):
+        k, v = K[l], V[l]
+        if k is None or k.shape[2] == 0:
+            arr[l] = mka_level(None, None, 0, 0, 0, 0)
+            continue
+        assert k.dim() == 4 and k.stride(3) == 1 and v.stride() == k.stride() and v.shape == k.shape
+        arr[l] = mka_level(k.data_ptr(), v.data_ptr(), k.shape[2], k.stride(0), k.stride(1), k.stride(2))
+    return arr
+
+
+def mka_workspace_bytes(shape: mka_shape, n_level, which: int) -> int:
+    return int(lib.mka_workspace_bytes(ctypes.byref(shape), _n_level(n_level), which))
+
+
+def mka_decode_plan(n_level, B: int, H: int, d: int):
+    plan = mka_decode_plan_t()
+    _check(lib.mka_decode_plan(_n_level(n_level), B, H, d, ctypes.byref(plan)), "mka_decode_plan")
+    return int(plan.chunk_rows), [int(x) for x in plan.n_chunks], int(plan.total_chunks)
+
+
+def mka_fwd_tile_range(shape: mka_shape, n_level, level: int, q_tile: int):
+    out = mka_tile_range()
+    _check(lib.mka_fwd_tile_range(ctypes.byref(shape), _n_level(n_level), level, q_tile, ctypes.byref(out)),
+           "mka_fwd_tile_range")
+    return int(out.first), int(out.end), int(out.full_first), int(out.full_end)
+
+
+def mka_router(R: torch.Tensor, W_r: torch.Tensor, b_r: Optional[torch.Tensor], route: int = MKA_ROUTE_SOFT,
+               gate: Optional[torch.Tensor] = None, log2_gate: Optional[torch.Tensor] = None,
+               route_idx: Optional[torch.Tensor] = None, stream=None):
+    """R[..., D] -> gate[..., 3] (f32).  Outputs may be preallocated; missing ones are allocated here."""
+    D = R.shape[-1]
+    rows = R.numel() // D if D else 0
+    assert R.is_contiguous() and W_r.is_contiguous() and W_r.dtype == torch.float32 and W_r.shape == (D, 3)
+    lead = tuple(R.shape[:-1])
+    if gate is None:
+        gate = torch.empty(lead + (3,), dtype=torch.float32, device=R.device)
+    _check(lib.mka_router(_ptr(R), _ptr(W_r), _ptr(b_r), rows, D, _dt(R), route, _ptr(gate), _ptr(log2_gate),
+                          _ptr(route_idx), _stream(stream)), "mka_router")
+    return gate
+
+
+def alloc_workspace(shape: mka_shape, n_level, which: int, device) -> torch.Tensor:
+    return torch.empty(mka_workspace_bytes(shape, n_level, which), dtype=torch.uint8, device=device)
+
+
+def mka_fwd(shape: mka_shape, Q, K, V, gate, O=None, LSE=None, ws=None, stream=None, want_lse=True):
+    assert Q.is_contiguous() and gate.is_contiguous() and gate.dtype == torch.float32
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None and want_lse and shape.mode == MKA_MODE_FAST:
+        LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device=Q.device)
+    n = [0 if k is None else k.shape[2] for k in K]
+    if ws is None:
+        ws = alloc_workspace(shape, n, MKA_WS_FWD, Q.device)
+    _check(lib.mka_fwd(ctypes.byref(shape), _ptr(Q), _levels(K, V), _ptr(gate), _ptr(O), _ptr(LSE), _ptr(ws),
+                       ws.numel(), _stream(stream)), "mka_fwd")
+    return O, LSE
+
+
+def mka_decode(shape: mka_shape, q, K, V, gate, O=None, LSE=None, ws=None, stream=None):
+    assert q.is_contiguous() and gate.is_contiguous() and gate.dtype == torch.float32
+    if O is None:
+        O = torch.empty_like(q)
+    if LSE is None:
+        LSE = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    n = [0 if k is None else k.shape[2] for k in K]
+    if ws is None:
+        ws = alloc_workspace(shape, n, MKA_WS_DECODE, q.device)
+    _check(lib.mka_decode(ctypes.byref(shape), _ptr(q), _levels(K, V), _ptr(gate), _ptr(O), _ptr(LSE), _ptr(ws),
+                          ws.numel(), _stream(stream)), "mka_decode")
+    return O, LSE
+
+
+def mka_bwd(shape: mka_shape, Q, K, V, gate, O, LSE, dO, R=None, dQ=None, dK=None, dV=None, dG=None, dW_r=None,
+            db_r=None, ws=None, stream=None, want_router_grad=True):
+    for t in (Q, O, dO, gate, LSE):
+        assert t.is_contiguous()
+    dev = Q.device
+    if dQ is None:
+        dQ = torch.empty_like(Q)
+    if dK is None:
+        dK = [None if k is None else torch.empty_like(k) for k in K]
+    if dV is None:
+        dV = [None if v is None else torch.empty_like(v) for v in V]
+    if dG is None:
+        dG = torch.empty(gate.shape, dtype=torch.float32, device=dev)
+    if R is not None and want_router_grad:
+        assert R.is_contiguous()
+        if dW_r is None:
+            dW_r = torch.empty((R.shape[-1], 3), dtype=torch.float32, device=dev)
+        if db_r is None:
+            db_r = torch.empty((3,), dtype=torch.float32, device=dev)
+    grads = (mka_level_grad * 3)()
+    for l in range(3):
+        if K[l] is None or K[l].shape[2] == 0:
+            grads[l] = mka_level_grad(None, None, 0, 0, 0, 0)
+        else:
+            g = dK[l]
+            assert g.stride(3) == 1 and dV[l].stride() == g.stride()
+            grads[l] = mka_level_grad(g.data_ptr(), dV[l].data_ptr(), g.shape[2], g.stride(0), g.stride(1), g.stride(2))
+    n = [0 if k is None else k.shape[2] for k in K]
+    if ws is None:
+        ws = alloc_workspace(shape, n, MKA_WS_BWD, dev)
+    _check(lib.mka_bwd(ctypes.byref(shape), _ptr(Q), _levels(K, V), _ptr(gate), _ptr(O), _ptr(LSE), _ptr(dO),
+                       _ptr(R), _dt(R) if R is not None else MKA_F32, _ptr(dQ), grads, _ptr(dG), _ptr(dW_r),
+                       _ptr(db_r), _ptr(ws), ws.numel(), _stream(stream)), "mka_bwd")
+    return {"dQ": dQ, "dK": dK, "dV": dV, "dG": dG, "dW_r": dW_r, "db_r": db_r}
+
+
+def mka_device_status(ws: torch.Tensor, stream=None) -> int:
+    return int(lib.mka_device_status(_ptr(ws), _stream(stream)))

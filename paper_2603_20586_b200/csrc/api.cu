@@ -1,0 +1,273 @@
+// C-ABI entry points of the FastMKA library: host-side validation, integer bookkeeping (decode split
+// table, forward tile ranges), workspace layout, and dispatch to the kernels.  See include/mka.h.
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace mka;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+mka_status check_shape(const mka_shape* s, bool decode) {
+    if (!s) return MKA_ERR_ARG;
+    if (s->dtype != MKA_BF16 && s->dtype != MKA_F32) return MKA_ERR_ARG;
+    if (s->mode != MKA_MODE_FAST && s->mode != MKA_MODE_FULL) return MKA_ERR_ARG;
+    if (s->B < 0 || s->H < 0 || s->T < 0) return MKA_ERR_SHAPE;
+    if (s->d != 32 && s->d != 64 && s->d != 96 && s->d != 128) return MKA_ERR_SHAPE;
+    if (!decode && s->window < 1) return MKA_ERR_SHAPE;
+    if (!decode && s->q_offset < 0) return MKA_ERR_SHAPE;
+    if (decode && s->T != 1) return MKA_ERR_SHAPE;
+    return MKA_OK;
+}
+
+mka_status check_levels(const mka_shape* s, const mka_level L[3]) {
+    if (!L) return MKA_ERR_ARG;
+    for (int l = 0; l < 3; ++l) {
+        if (L[l].n < 0) return MKA_ERR_SHAPE;
+        if (L[l].n == 0) continue;
+        if (!L[l].k || !L[l].v) return MKA_ERR_ARG;
+        if (L[l].stride_n < s->d || L[l].stride_b < 0 || L[l].stride_h < 0) return MKA_ERR_SHAPE;
+        if (s->dtype == MKA_BF16) {
+            if (!aligned16(L[l].k) || !aligned16(L[l].v)) return MKA_ERR_ALIGN;
+            if (L[l].stride_n % 8 || L[l].stride_b % 8 || L[l].stride_h % 8) return MKA_ERR_ALIGN;
+        }
+    }
+    return MKA_OK;
+}
+
+float resolve_scale(const mka_shape* s) { return s->scale > 0.f ? s->scale : 1.0f / sqrtf((float)s->d); }
+
+void fill_levels(LevelDev out[3], const mka_level L[3]) {
+    for (int l = 0; l < 3; ++l) {
+        out[l].k = L[l].k; out[l].v = L[l].v; out[l].n = L[l].n;
+        out[l].sb = L[l].stride_b; out[l].sh = L[l].stride_h; out[l].sn = L[l].stride_n;
+    }
+}
+
+constexpr int kRouterBwdChunks = 128;
+
+}  // namespace
+
+extern "C" {
+
+const char* mka_status_str(mka_status s) {
+    switch (s) {
+        case MKA_OK: return "ok";
+        case MKA_ERR_ARG: return "invalid argument";
+        case MKA_ERR_SHAPE: return "invalid shape";
+        case MKA_ERR_ALIGN: return "misaligned pointer or stride";
+        case MKA_ERR_WORKSPACE: return "workspace missing or too small";
+        case MKA_ERR_UNSUPPORTED: return "unsupported combination";
+        case MKA_ERR_CUDA: return "CUDA runtime error";
+        case MKA_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+mka_status mka_decode_plan(const int64_t n_level[3], int32_t B, int32_t H, int32_t d, mka_decode_plan_t* plan) {
+    if (!n_level || !plan) return MKA_ERR_ARG;
+    if (B < 0 || H < 0 || d <= 0) return MKA_ERR_SHAPE;
+    int64_t total_rows = 0;
+    for (int l = 0; l < 3; ++l) {
+        if (n_level[l] < 0) return MKA_ERR_SHAPE;
+        total_rows += n_level[l];
+    }
+    // Aim for at least ~8 CTAs per SM over the whole grid, with chunks of 128..1024 rows (multiples of
+    // 128) so that every CTA streams the same number of bytes apart from each level's last chunk.
+    const int64_t target_ctas = 148 * 8;
+    const int64_t bh = (int64_t)B * H > 0 ? (int64_t)B * H : 1;
+    int64_t rows = (total_rows * bh + target_ctas - 1) / target_ctas;   // rows per CTA to hit the target
+    rows = (rows / 128) * 128;
+    if (rows < 128) rows = 128;
+    if (rows > 1024) rows = 1024;
+    plan->chunk_rows = rows;
+    plan->total_chunks = 0;
+    for (int l = 0; l < 3; ++l) {
+        plan->n_chunks[l] = (n_level[l] + rows - 1) / rows;
+        plan->total_chunks += plan->n_chunks[l];
+    }
+    return MKA_OK;
+}
+
+mka_status mka_fwd_tile_range(const mka_shape* s, const int64_t n_level[3], int32_t level, int64_t q_tile,
+                              mka_tile_range* out) {
+    if (!s || !n_level || !out) return MKA_ERR_ARG;
+    if (level < 0 || level > 2 || q_tile < 0 || q_tile * kTileM >= (s->T > 0 ? s->T : 1)) return MKA_ERR_SHAPE;
+    const long long n = n_level[level], W = s->window;
+    const long long m0 = q_tile * kTileM;
+    const long long m1 = (m0 + kTileM - 1 < s->T - 1 ? m0 + kTileM - 1 : s->T - 1);
+    const long long p_lo = m0 + s->q_offset, p_hi = m1 + s->q_offset;
+    long long lo_f, hi_f, lo_l, hi_l;
+    visible_range(level, p_lo, W, n, 0, lo_f, hi_f);
+    visible_range(level, p_hi, W, n, 0, lo_l, hi_l);
+    const long long lo = lo_f, hi = hi_l > hi_f ? hi_l : hi_f;     // union (ranges move right with p)
+    if (hi <= lo) { out->first = out->end = out->full_first = out->full_end = 0; return MKA_OK; }
+    out->first = lo / kTileN;
+    out->end = (hi + kTileN - 1) / kTileN;
+    // intersection of all rows' ranges: [lo_l, hi_f); a key tile is "full" when it lies inside it
+    const long long ilo = lo_l, ihi = hi_f;
+    long long ff = (ilo + kTileN - 1) / kTileN, fe = ihi / kTileN;
+    if (ff < out->first) ff = out->first;
+    if (fe > out->end) fe = out->end;
+    if (fe < ff) fe = ff;
+    out->full_first = ff;
+    out->full_end = fe;
+    return MKA_OK;
+}
+
+size_t mka_workspace_bytes(const mka_shape* s, const int64_t n_level[3], int32_t which) {
+    if (!s || !n_level) return 0;
+    if (which == MKA_WS_FWD) return kWsHeader;
+    if (which == MKA_WS_DECODE) {
+        mka_decode_plan_t plan;
+        if (mka_decode_plan(n_level, s->B, s->H, s->d, &plan) != MKA_OK) return 0;
+        return kWsHeader + round_up((size_t)s->B * s->H * plan.total_chunks * (s->d + 2) * sizeof(float), 256);
+    }
+    if (which == MKA_WS_BWD) {
+        size_t rows = (size_t)s->B * s->H * s->T;
+        return kWsHeader + round_up(rows * sizeof(float), 256) + round_up(rows * 3 * sizeof(float), 256) +
+               round_up((size_t)kRouterBwdChunks * (s->D > 0 ? s->D : 0) * 3 * sizeof(float), 256);
+    }
+    return 0;
+}
+
+mka_status mka_router(const void* R, const float* W_r, const float* b_r, int64_t rows, int32_t D, int32_t r_dtype,
+                      int32_t route, float* gate, float* log2_gate, int8_t* route_idx, void* stream) {
+    if (rows < 0 || D <= 0) return MKA_ERR_SHAPE;
+    if (r_dtype != MKA_BF16 && r_dtype != MKA_F32) return MKA_ERR_ARG;
+    if (route < MKA_ROUTE_SOFT || route > MKA_ROUTE_TOP2) return MKA_ERR_ARG;
+    if (rows == 0) return MKA_OK;
+    if (!R || !W_r || !gate) return MKA_ERR_ARG;
+    cudaError_t e = launch_router(R, W_r, b_r, rows, D, r_dtype, route, gate, log2_gate, route_idx,
+                                  static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
+mka_status mka_fwd(const mka_shape* s, const void* Q, const mka_level L[3], const float* gate, void* O, float* LSE,
+                   void* ws, size_t ws_bytes, void* stream) {
+    mka_status st = check_shape(s, false);
+    if (st != MKA_OK) return st;
+    if ((st = check_levels(s, L)) != MKA_OK) return st;
+    if (s->B == 0 || s->H == 0 || s->T == 0) return MKA_OK;
+    if (!Q || !gate || !O) return MKA_ERR_ARG;
+    if (s->dtype == MKA_BF16 && (!aligned16(Q) || !aligned16(O))) return MKA_ERR_ALIGN;
+    if (!ws || ws_bytes < kWsHeader) return MKA_ERR_WORKSPACE;
+    FwdParams p;
+    memset(&p, 0, sizeof(p));
+    p.Q = Q; p.O = O; p.LSE = LSE; p.gate = gate;
+    fill_levels(p.L, L);
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
+    p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s);
+    p.mode = s->mode; p.decode = 0;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
+    cudaError_t e;
+    if (!(s->flags & MKA_FLAG_FORCE_SIMT) && s->mode == MKA_MODE_FAST && fwd_tc_eligible(p, s->dtype))
+        e = launch_fwd_tc(p, static_cast<unsigned int*>(ws), cs);
+    else
+        e = launch_fwd_simt(p, s->dtype, cs);
+    if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
+mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], const float* gate, void* O,
+                      float* LSE, void* ws, size_t ws_bytes, void* stream) {
+    mka_status st = check_shape(s, true);
+    if (st != MKA_OK) return st;
+    if (s->dtype != MKA_BF16 || s->mode != MKA_MODE_FAST) return MKA_ERR_UNSUPPORTED;
+    if (s->d != 64 && s->d != 128) return MKA_ERR_SHAPE;
+    if ((st = check_levels(s, L)) != MKA_OK) return st;
+    if (s->B == 0 || s->H == 0) return MKA_OK;
+    if (!q || !gate || !O) return MKA_ERR_ARG;
+    if (!aligned16(q) || !aligned16(O)) return MKA_ERR_ALIGN;
+    int64_t n_level[3] = {L[0].n, L[1].n, L[2].n};
+    size_t need = mka_workspace_bytes(s, n_level, MKA_WS_DECODE);
+    if (!ws || ws_bytes < need) return MKA_ERR_WORKSPACE;
+    mka_decode_plan_t plan;
+    mka_decode_plan(n_level, s->B, s->H, s->d, &plan);
+    if ((long long)s->B * s->H * plan.total_chunks > 0x7fffffffLL) return MKA_ERR_SHAPE;
+    DecodeParams p;
+    memset(&p, 0, sizeof(p));
+    p.q = q; p.O = O; p.LSE = LSE; p.gate = gate;
+    fill_levels(p.L, L);
+    p.B = s->B; p.H = s->H; p.d = s->d; p.scale = resolve_scale(s);
+    p.chunk_rows = plan.chunk_rows;
+    for (int l = 0; l < 3; ++l) p.n_chunks[l] = plan.n_chunks[l];
+    p.total_chunks = plan.total_chunks;
+    p.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeader);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
+    cudaError_t e = launch_decode(p, cs);
+    if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
+mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], const float* gate, const void* O,
+                   const float* LSE, const void* dO, const void* R, int32_t r_dtype, void* dQ,
+                   const mka_level_grad dL[3], float* dG, float* dW_r, float* db_r, void* ws, size_t ws_bytes,
+                   void* stream) {
+    mka_status st = check_shape(s, false);
+    if (st != MKA_OK) return st;
+    if (s->mode != MKA_MODE_FAST) return MKA_ERR_UNSUPPORTED;
+    if ((st = check_levels(s, L)) != MKA_OK) return st;
+    if (!dL) return MKA_ERR_ARG;
+    for (int l = 0; l < 3; ++l) {
+        if (dL[l].n != L[l].n) return MKA_ERR_SHAPE;
+        if (L[l].n == 0) continue;
+        if (!dL[l].dk || !dL[l].dv) return MKA_ERR_ARG;
+        if (dL[l].stride_n < s->d) return MKA_ERR_SHAPE;
+        if (s->dtype == MKA_BF16 && (!aligned16(dL[l].dk) || !aligned16(dL[l].dv) || dL[l].stride_n % 8 ||
+                                     dL[l].stride_b % 8 || dL[l].stride_h % 8))
+            return MKA_ERR_ALIGN;
+    }
+    if ((dW_r || db_r) && r_dtype != MKA_BF16 && r_dtype != MKA_F32) return MKA_ERR_ARG;
+    if (dW_r && (!R || s->D <= 0)) return MKA_ERR_ARG;
+    if (s->B == 0 || s->H == 0 || s->T == 0) return MKA_OK;
+    if (!Q || !gate || !O || !LSE || !dO || !dQ || !dG) return MKA_ERR_ARG;
+    if (s->dtype == MKA_BF16 && (!aligned16(Q) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ))) return MKA_ERR_ALIGN;
+    int64_t n_level[3] = {L[0].n, L[1].n, L[2].n};
+    size_t need = mka_workspace_bytes(s, n_level, MKA_WS_BWD);
+    if (!ws || ws_bytes < need) return MKA_ERR_WORKSPACE;
+    const size_t rows = (size_t)s->B * s->H * s->T;
+    char* w = static_cast<char*>(ws) + kWsHeader;
+    BwdParams p;
+    memset(&p, 0, sizeof(p));
+    p.Q = Q; p.O = O; p.dO = dO; p.LSE = LSE; p.gate = gate; p.dQ = dQ; p.dG = dG;
+    fill_levels(p.L, L);
+    for (int l = 0; l < 3; ++l) {
+        p.dL[l].dk = dL[l].dk; p.dL[l].dv = dL[l].dv; p.dL[l].n = dL[l].n;
+        p.dL[l].sb = dL[l].stride_b; p.dL[l].sh = dL[l].stride_h; p.dL[l].sn = dL[l].stride_n;
+    }
+    p.delta = reinterpret_cast<float*>(w);
+    w += round_up(rows * sizeof(float), 256);
+    p.Gpart = reinterpret_cast<float*>(w);
+    w += round_up(rows * 3 * sizeof(float), 256);
+    float* rpart = reinterpret_cast<float*>(w);
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
+    p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
+    cudaError_t e = launch_bwd_simt(p, s->dtype, cs);
+    if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return MKA_ERR_CUDA;
+    if (dW_r || db_r) {
+        e = launch_router_bwd(R, r_dtype, dG, (long long)s->B * s->T, s->D, dW_r, db_r, rpart, kRouterBwdChunks, cs);
+        if (e != cudaSuccess) return MKA_ERR_CUDA;
+    }
+    return MKA_OK;
+}
+
+mka_status mka_device_status(const void* ws, void* stream) {
+    if (!ws) return MKA_ERR_ARG;
+    unsigned int word = 0;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return MKA_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return MKA_ERR_CUDA;
+    return word == 0 ? MKA_OK : MKA_ERR_TIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,125 @@
+// Internal declarations shared by the kernels of the FastMKA library (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "mka.h"
+
+namespace mka {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kTileM = 128;   // query rows per tile of the tensor-core forward
+constexpr int kTileN = 128;   // key rows per tile
+
+// Layout of the caller's workspace: a 256-byte header (device status word first), then the
+// per-entry-point scratch.
+constexpr size_t kWsHeader = 256;
+
+struct LevelDev {
+    const void* k;
+    const void* v;
+    long long n, sb, sh, sn;
+};
+
+struct LevelGradDev {
+    void* dk;
+    void* dv;
+    long long n, sb, sh, sn;
+};
+
+struct FwdParams {
+    const void* Q;
+    void* O;
+    float* LSE;         // may be null
+    const float* gate;  // [B,T,3]
+    LevelDev L[3];
+    int B, H, T, d;
+    int window, q_offset;
+    float scale;        // tau
+    int mode;
+    int decode;         // every row visible
+};
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static __device__ __forceinline__ float ld(const float* p) { return *p; }
+    static __device__ __forceinline__ void st(float* p, float v) { *p = v; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static __device__ __forceinline__ float ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+// Rows [lo, hi) of `level` visible to key-timeline position p (L1 causal window, L2 causal prefix,
+// L3 everything), clipped to [0, n).
+__host__ __device__ __forceinline__ void visible_range(int level, long long p, long long W, long long n,
+                                                       int decode, long long& lo, long long& hi) {
+    long long a = 0, b = n;
+    if (!decode) {
+        if (level == 0) { a = p - W + 1; b = p + 1; }
+        else if (level == 1) { b = p + 1; }
+        if (a < 0) a = 0;
+        if (b > n) b = n;
+    }
+    if (b < a) b = a;
+    lo = a; hi = b;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---- launchers implemented in the .cu files (all return a cudaError_t from the launch) ----
+cudaError_t launch_router(const void* R, const float* W_r, const float* b_r, long long rows, int D, int r_dtype,
+                          int route, float* gate, float* log2_gate, int8_t* idx, cudaStream_t st);
+cudaError_t launch_fwd_simt(const FwdParams& p, int dtype, cudaStream_t st);
+
+struct DecodeParams {
+    const void* q;
+    void* O;
+    float* LSE;
+    const float* gate;   // [B,3]
+    LevelDev L[3];
+    int B, H, d;
+    float scale;
+    long long chunk_rows;
+    long long n_chunks[3];
+    long long total_chunks;
+    float* partial;      // [B*H, total_chunks, d+2]
+};
+cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st);
+
+struct BwdParams {
+    const void *Q, *O, *dO;
+    const float* LSE;
+    const float* gate;
+    LevelDev L[3];
+    LevelGradDev dL[3];
+    void* dQ;
+    float* dG;        // [B,T,3]
+    float* delta;     // ws: [B,H,T]
+    float* Gpart;     // ws: [B,H,T,3]
+    int B, H, T, d;
+    int window, q_offset;
+    float scale;
+};
+cudaError_t launch_bwd_simt(const BwdParams& p, int dtype, cudaStream_t st);
+cudaError_t launch_router_bwd(const void* R, int r_dtype, const float* dG, long long rows, int D, float* dW_r,
+                              float* db_r, float* partial, int n_row_chunks, cudaStream_t st);
+
+// Tensor-core (TMA + tcgen05) forward; returns cudaErrorNotSupported when the shape is not eligible.
+cudaError_t launch_fwd_tc(const FwdParams& p, unsigned int* status_word, cudaStream_t st);
+bool fwd_tc_eligible(const FwdParams& p, int dtype);
+
+}  // namespace mka

@@ -1,0 +1,260 @@
+"""GPU parity: every entry point of the C ABI against the CPU oracle, element by element, on seeded
+inputs small enough for the oracle to finish in seconds but spanning several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_helpers import check, err, np64, problem
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mka():
+    import paper_2603_20586_b200 as m
+    assert torch.cuda.is_available()
+    return m
+
+
+def _dt(mka, dtype):
+    return mka.binding.MKA_BF16 if dtype == torch.bfloat16 else mka.binding.MKA_F32
+
+
+# ------------------------------------------------------------------ router
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("rows,D", [(256, 256), (37, 1024), (5, 100), (1, 8), (1000, 4096)])
+def test_router_soft(mka, orc, dtype, rows, D):
+    X = problem(5, 1, 1, rows, 32, (1, 1, 1), D, dtype)["X"].view(rows, D)
+    W = torch.randn(D, 3, device="cuda") * 0.05
+    b = torch.tensor([0.1, -0.2, 0.05], device="cuda")
+    log2g = torch.empty(rows, 3, device="cuda")
+    idx = torch.full((rows, 2), 7, dtype=torch.int8, device="cuda")
+    gate = mka.mka_router(X, W, b, log2_gate=log2g, route_idx=idx)
+    ref, _ = orc.router(np64(X), np64(W), np64(b))
+    mx, _ = err(gate, ref)
+    assert mx <= 2e-6
+    assert err(gate.sum(-1), np.ones(rows))[0] <= 1e-6
+    assert err(log2g, np.log2(ref))[0] <= 1e-5
+    assert (idx == -1).all()
+    g0 = mka.mka_router(X, W, None)
+    assert err(g0, orc.router(np64(X), np64(W), None)[0])[0] <= 2e-6
+
+
+def test_router_topk_indices_bit_exact_on_exact_logits(mka, orc):
+    # integer-valued inputs make every logit exact in fp32 and fp64, so ties and orderings are decided
+    # identically: kept indices must match bit for bit.
+    g = torch.Generator().manual_seed(3)
+    rows, D = 4096, 16
+    X = torch.randint(-2, 3, (rows, D), generator=g).float().cuda()
+    W = torch.randint(-1, 2, (D, 3), generator=g).float().cuda()
+    for route in (mka.binding.MKA_ROUTE_TOP1, mka.binding.MKA_ROUTE_TOP2, mka.binding.MKA_ROUTE_UNIFORM):
+        idx = torch.empty(rows, 2, dtype=torch.int8, device="cuda")
+        gate = mka.mka_router(X, W, None, route=route, route_idx=idx)
+        ref, ridx = orc.router(np64(X), np64(W), None, route=route)
+        assert np.array_equal(idx.cpu().numpy(), ridx)
+        assert err(gate, ref)[0] <= 2e-6
+        assert np.array_equal(gate.cpu().numpy() == 0, ref == 0)
+
+
+def test_router_topk_random_logits(mka, orc):
+    P = problem(9, 2, 1, 500, 32, (1, 1, 1), 256, torch.bfloat16, router_std=1.0)
+    X, W = P["X"], P["W_r"]
+    idx = torch.empty(2, 500, 2, dtype=torch.int8, device="cuda")
+    gate = mka.mka_router(X, W, None, route=mka.binding.MKA_ROUTE_TOP2, route_idx=idx)
+    ref, ridx = orc.router(np64(X), np64(W), None, route=orc.ROUTE_TOP2)
+    logits = np64(X) @ np64(W)
+    diff = (idx.cpu().numpy() != ridx).any(-1)
+    # a disagreement is only legitimate where the two candidate logits are within fp32 rounding of each other
+    for b, t in zip(*np.nonzero(diff)):
+        s = np.sort(logits[b, t])
+        assert min(s[1] - s[0], s[2] - s[1]) < 1e-4
+    ok = ~diff
+    assert err(gate[torch.from_numpy(ok).cuda()], ref[ok])[0] <= 5e-6
+
+
+# ------------------------------------------------------------------ forward
+FWD_CASES = [
+    # B, H, T, d, W, q_off, N
+    (1, 2, 200, 64, 64, 0, (200, 200, 130)),        # ragged T, ragged N3
+    (2, 1, 256, 128, 512, 0, (256, 256, 0)),        # W > T (plain causal), no L3 (Local-MKA)
+    (1, 2, 130, 64, 100, 700, (830, 830, 257)),     # cached prefix: q_offset > 0
+    (1, 1, 1, 128, 1, 0, (1, 1, 1)),                # single row
+    (1, 3, 384, 128, 129, 3, (387, 300, 128)),      # N2 shorter than the timeline
+    (1, 1, 96, 64, 32, 0, (96, 0, 40)),             # no L2
+]
+
+
+@pytest.mark.parametrize("case", FWD_CASES)
+@pytest.mark.parametrize("dtype,flags", [(torch.bfloat16, 0), (torch.bfloat16, 1), (torch.float32, 0)])
+def test_fwd_fast_matches_oracle(mka, orc, case, dtype, flags):
+    B, H, T, d, W, q_off, N = case
+    P = problem(11, B, H, T, d, N, 64, dtype, router_std=0.3)
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    shape = mka.make_shape(B, H, T, d, 64, W, q_off, dtype=_dt(mka, dtype), flags=flags)
+    O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+    torch.cuda.synchronize()
+    rg, _ = orc.router(np64(P["X"]), np64(P["W_r"]))
+    Or, Lr = orc.fwd(P["Q"], P["K"], P["V"], rg, W, q_off)
+    check(O, Or, dtype, "O")
+    assert err(LSE, Lr)[0] <= (1e-4 if dtype == torch.float32 else 2e-3)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fwd_full_mode_matches_alg1_oracle(mka, orc, dtype):
+    B, H, T, d, W, N = 1, 2, 150, 64, 40, (150, 150, 70)
+    P = problem(13, B, H, T, d, N, 32, dtype, router_std=0.5)
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    shape = mka.make_shape(B, H, T, d, 32, W, dtype=_dt(mka, dtype), mode=mka.binding.MKA_MODE_FULL)
+    O, _ = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+    rg, _ = orc.router(np64(P["X"]), np64(P["W_r"]))
+    Or, _ = orc.fwd(P["Q"], P["K"], P["V"], rg, W, mode="full")
+    check(O, Or, dtype, "O full")
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_fwd_one_hot_and_topk_gates(mka, orc, flags):
+    B, H, T, d, W, N = 1, 2, 260, 128, 70, (260, 260, 140)
+    P = problem(17, B, H, T, d, N, 32, torch.bfloat16, router_std=1.0)
+    shape = mka.make_shape(B, H, T, d, 32, W, flags=flags)
+    for l in range(3):
+        gate = torch.zeros(B, T, 3, device="cuda")
+        gate[..., l] = 1.0
+        O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+        Or, Lr = orc.fwd(P["Q"], P["K"], P["V"], np64(gate), W)
+        check(O, Or, torch.bfloat16, f"one-hot {l}")
+        assert err(LSE, Lr)[0] <= 2e-3
+    gate = mka.mka_router(P["X"], P["W_r"], None, route=mka.binding.MKA_ROUTE_TOP1)
+    O, _ = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+    rg, _ = orc.router(np64(P["X"]), np64(P["W_r"]), route=orc.ROUTE_TOP1)
+    assert np.array_equal(gate.cpu().numpy() == 0, rg == 0)
+    check(O, orc.fwd(P["Q"], P["K"], P["V"], rg, W)[0], torch.bfloat16, "top-1")
+
+
+def test_fwd_nothing_visible_rows_are_zero(mka):
+    B, H, T, d = 1, 1, 140, 64
+    P = problem(19, B, H, T, d, (0, 0, 50), 16, torch.bfloat16)
+    gate = torch.zeros(B, T, 3, device="cuda")
+    gate[..., 0] = 1.0                                   # all weight on an empty level
+    for flags in (0, 1):
+        shape = mka.make_shape(B, H, T, d, 16, 8, flags=flags)
+        O, LSE = mka.mka_fwd(shape, P["Q"], [None, None, P["K"][2]], [None, None, P["V"][2]], gate)
+        assert (O == 0).all() and torch.isneginf(LSE).all()
+
+
+def test_fwd_strided_levels(mka, orc):
+    # levels stored as slices of a bigger cache: explicit batch/head/row strides
+    B, H, T, d, W = 1, 2, 192, 64, 50
+    P = problem(23, B, H, T, d, (T, T, 64), 16, torch.bfloat16)
+    big = [torch.zeros(B, H, k.shape[2] + 16, 2 * d, dtype=torch.bfloat16, device="cuda") for k in P["K"]]
+    Ks, Vs = [], []
+    for l in range(3):
+        n = P["K"][l].shape[2]
+        big[l][:, :, 8:8 + n, :d] = P["K"][l]
+        big[l][:, :, 8:8 + n, d:] = P["V"][l]
+        Ks.append(big[l][:, :, 8:8 + n, :d])
+        Vs.append(big[l][:, :, 8:8 + n, d:])
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    for flags in (0, 1):
+        shape = mka.make_shape(B, H, T, d, 16, W, flags=flags)
+        O, _ = mka.mka_fwd(shape, P["Q"], Ks, Vs, gate)
+        Or, _ = orc.fwd(P["Q"], P["K"], P["V"], np64(gate), W)
+        check(O, Or, torch.bfloat16, "strided")
+
+
+# ------------------------------------------------------------------ decode
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("B,H,N", [(2, 3, (300, 1000, 77)), (1, 2, (0, 2500, 0)), (3, 1, (129, 1, 4100))])
+def test_decode_matches_oracle(mka, orc, d, B, H, N):
+    P = problem(29, B, H, 1, d, N, 64, torch.bfloat16, router_std=0.5)
+    gate = mka.mka_router(P["X"], P["W_r"], None).view(B, 3)
+    q = P["Q"].view(B, H, d)
+    shape = mka.make_shape(B, H, 1, d, 64)
+    K = [k if k.shape[2] else None for k in P["K"]]
+    V = [v if v.shape[2] else None for v in P["V"]]
+    O, LSE = mka.mka_decode(shape, q, K, V, gate)
+    Or, Lr = orc.fwd(P["Q"], P["K"], P["V"], np64(gate).reshape(B, 1, 3), 1, decode=True)
+    check(O.view(B, H, 1, d), Or, torch.bfloat16, "decode O")
+    assert err(LSE.view(B, H, 1), Lr)[0] <= 2e-3
+
+
+def test_decode_equals_last_prefill_row_and_zero_gate_level(mka, orc):
+    B, H, T, d, W = 1, 2, 300, 128, 100
+    P = problem(31, B, H, T, d, (T, T, 90), 32, torch.bfloat16)
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    O, _ = mka.mka_fwd(mka.make_shape(B, H, T, d, 32, W), P["Q"], P["K"], P["V"], gate)
+    t = T - 1
+    Kd = [P["K"][0][:, :, t - W + 1:t + 1].contiguous(), P["K"][1], P["K"][2]]
+    Vd = [P["V"][0][:, :, t - W + 1:t + 1].contiguous(), P["V"][1], P["V"][2]]
+    q = P["Q"][:, :, t].contiguous()
+    g = gate[:, t].contiguous()
+    Od, _ = mka.mka_decode(mka.make_shape(B, H, 1, d, 32), q, Kd, Vd, g)
+    assert (Od.float() - O[:, :, t].float()).abs().max().item() <= 2e-2
+    g0 = g.clone()
+    g0[:, 1] = 0.0
+    g0 /= g0.sum(-1, keepdim=True)
+    Oz, Lz = mka.mka_decode(mka.make_shape(B, H, 1, d, 32), q, Kd, Vd, g0)
+    Or, Lr = orc.fwd(q.view(B, H, 1, d), Kd, Vd, np64(g0).reshape(B, 1, 3), 1, decode=True)
+    check(Oz.view(B, H, 1, d), Or, torch.bfloat16, "decode zero-gate level")
+
+
+# ------------------------------------------------------------------ backward
+BWD_CASES = [
+    (1, 2, 200, 64, 64, 0, (200, 200, 130)),
+    (2, 2, 96, 128, 200, 0, (96, 96, 0)),
+    (1, 1, 70, 64, 30, 50, (120, 120, 33)),
+]
+
+
+@pytest.mark.parametrize("case", BWD_CASES)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_bwd_matches_oracle(mka, orc, case, dtype):
+    B, H, T, d, W, q_off, N = case
+    D = 48
+    P = problem(37, B, H, T, d, N, D, dtype, router_std=0.3, with_dO=True)
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    shape = mka.make_shape(B, H, T, d, D, W, q_off, dtype=_dt(mka, dtype))
+    O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+    K = [k if k.shape[2] else None for k in P["K"]]
+    V = [v if v.shape[2] else None for v in P["V"]]
+    g = mka.mka_bwd(shape, P["Q"], K, V, gate, O, LSE, P["dO"], R=P["X"])
+    torch.cuda.synchronize()
+    rg, _ = orc.router(np64(P["X"]), np64(P["W_r"]))
+    ref = orc.bwd(P["Q"], P["K"], P["V"], rg, P["dO"], W, q_off)
+    check(g["dQ"], ref["dQ"], dtype, "dQ")
+    for l in range(3):
+        if N[l]:
+            check(g["dK"][l], ref["dK"][l], dtype, f"dK{l}")
+            check(g["dV"][l], ref["dV"][l], dtype, f"dV{l}")
+    # dG sums H heads of fp32 partials; gradients w.r.t. logits are small numbers
+    tol = 2e-2 if dtype == torch.bfloat16 else 1e-4
+    assert err(g["dG"], ref["dG"])[0] <= tol
+    assert abs(float(g["dG"].sum(-1).abs().max())) <= tol            # sum_l dG_l = 0
+    dW, db = orc.router_bwd(np64(P["X"]), ref["dG"])
+    scale = max(1.0, float(np.abs(dW).max()))
+    assert err(g["dW_r"], dW)[0] <= (5e-2 if dtype == torch.bfloat16 else 2e-4) * scale
+    assert err(g["db_r"], db)[0] <= (5e-2 if dtype == torch.bfloat16 else 2e-4) * max(1.0, float(np.abs(db).max()))
+
+
+def test_bwd_is_deterministic(mka):
+    B, H, T, d, W, N = 1, 2, 160, 64, 40, (160, 160, 50)
+    P = problem(41, B, H, T, d, N, 32, torch.bfloat16, with_dO=True)
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    shape = mka.make_shape(B, H, T, d, 32, W)
+    O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+    a = mka.mka_bwd(shape, P["Q"], P["K"], P["V"], gate, O, LSE, P["dO"], R=P["X"])
+    b = mka.mka_bwd(shape, P["Q"], P["K"], P["V"], gate, O, LSE, P["dO"], R=P["X"])
+    for k in ("dQ", "dG", "dW_r"):
+        assert torch.equal(a[k], b[k])
+    for l in range(3):
+        assert torch.equal(a["dK"][l], b["dK"][l]) and torch.equal(a["dV"][l], b["dV"][l])
+
+
+def test_workspace_too_small_is_rejected(mka):
+    B, H, d = 1, 1, 128
+    q = torch.zeros(B, H, d, dtype=torch.bfloat16, device="cuda")
+    K = torch.zeros(B, H, 256, d, dtype=torch.bfloat16, device="cuda")
+    gate = torch.full((B, 3), 1 / 3, device="cuda")
+    ws = torch.empty(300, dtype=torch.uint8, device="cuda")
+    with pytest.raises(mka.MkaError) as e:
+        mka.mka_decode(mka.make_shape(B, H, 1, d), q, [K, None, None], [K, None, None], gate, ws=ws)
+    assert e.value.code == 4
