@@ -176,6 +176,10 @@ mka_status mka_decode_plan(const int64_t n_level[3], int32_t B, int32_t H, int32
 mka_status mka_fwd_tile_range(const mka_shape* shape, const int64_t n_level[3], int32_t level,
                               int64_t q_tile, mka_tile_range* out);
 
+/* Which forward kernel mka_fwd would run for this problem (host function, no launch):
+ * 0 = CUDA-core kernel, 1 = TMA + tcgen05 tensor-core kernel, negative = arguments invalid. */
+int32_t mka_fwd_kernel_kind(const mka_shape* shape, const mka_level L[3]);
+
 /* Synchronises `stream` and returns the device status word that the kernels of the last call using
  * `ws` left there: MKA_OK, or MKA_ERR_TIMEOUT when a bounded wait inside a kernel gave up (the
  * kernel then released its resources and returned; outputs of that call are invalid). */

@@ -23,7 +23,7 @@ MKA_WS_FWD, MKA_WS_DECODE, MKA_WS_BWD = 0, 1, 2
 TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
-           "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status"]
+           "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind"]
 
 
 class MkaError(RuntimeError):
@@ -77,6 +77,7 @@ def _load() -> ctypes.CDLL:
     lib.mka_fwd_tile_range.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(ctypes.c_int64), i32, i64,
                                        ctypes.POINTER(mka_tile_range)]
     lib.mka_device_status.argtypes = [vp, vp]
+    lib.mka_fwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level)]
     for name in EXPORTS:
         if name not in ("mka_status_str", "mka_workspace_bytes"):
             getattr(lib, name).restype = ctypes.c_int
@@ -231,6 +232,10 @@ def mka_bwd(shape: mka_shape, Q, K, V, gate, O, LSE, dO, R=None, dQ=None, dK=Non
                        _ptr(R), _dt(R) if R is not None else MKA_F32, _ptr(dQ), grads, _ptr(dG), _ptr(dW_r),
                        _ptr(db_r), _ptr(ws), ws.numel(), _stream(stream)), "mka_bwd")
     return {"dQ": dQ, "dK": dK, "dV": dV, "dG": dG, "dW_r": dW_r, "db_r": db_r}
+
+
+def mka_fwd_kernel_kind(shape: mka_shape, K, V) -> int:
+    return int(lib.mka_fwd_kernel_kind(ctypes.byref(shape), _levels(K, V)))
 
 
 def mka_device_status(ws: torch.Tensor, stream=None) -> int:

@@ -174,6 +174,15 @@ mka_status mka_fwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
 }
 
+int32_t mka_fwd_kernel_kind(const mka_shape* s, const mka_level L[3]) {
+    if (check_shape(s, false) != MKA_OK || check_levels(s, L) != MKA_OK) return -1;
+    FwdParams p;
+    memset(&p, 0, sizeof(p));
+    fill_levels(p.L, L);
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.mode = s->mode;
+    return (!(s->flags & MKA_FLAG_FORCE_SIMT) && s->mode == MKA_MODE_FAST && fwd_tc_eligible(p, s->dtype)) ? 1 : 0;
+}
+
 mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], const float* gate, void* O,
                       float* LSE, void* ws, size_t ws_bytes, void* stream) {
     mka_status st = check_shape(s, true);

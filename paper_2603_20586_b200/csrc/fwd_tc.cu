@@ -1,6 +1,528 @@
-// placeholder until the tensor-core forward lands
+// Tensor-core forward of Eq. 5 for bf16 on sm_100a: TMA -> shared memory -> tcgen05.mma -> TMEM.
+//
+// One CTA owns 256 query rows (two 128-row tiles, "ping" and "pong") of one (batch, head) and walks
+// ONE level-ordered list of 128-row key tiles: all visible L1 tiles, then L2, then L3.  A single
+// running (max, sum) per row spans the three levels (the max shift of Eq. 11-14); the gate enters
+// as a per-row, per-level additive bias log2(lambda) inside the exponent, so that
+//     p = 2^(s * tau * log2(e) + log2(lambda_l) - m)  =  lambda_l * exp(s*tau - m')
+// which is exactly the gated, un-normalised weight of Eq. 5.  One normalisation at the end.
+//
+// Warp roles (320 threads):
+//   warps 0-3 / 4-7  softmax warpgroup of query tile 0 / 1: thread i <-> TMEM lane i <-> query row i.
+//                    Reads S from TMEM, applies bias and masks, running max, exp2, writes P (bf16)
+//                    back into the TMEM columns S occupied, rescales the O accumulator when the
+//                    running maximum grows by more than 2^8 (lazy rescale), and does the epilogue.
+//   warp 8           producer: one lane issues the TMA loads of Q and of the K / V tile list into
+//                    128-byte-swizzled shared-memory rings (one mbarrier pair per stage).
+//   warp 9           one lane issues every tcgen05.mma: S_q = Q_q K^T (both operands from shared
+//                    memory) and O_q += P_q V (P from TMEM, V from shared memory, N-major), in the
+//                    order  S0(e)  O1(e-1)  S1(e)  O0(e)  so that each warpgroup's softmax overlaps
+//                    the other tile's matrix products.
+// TMEM: columns [0,128) S0/P0, [128,256) S1/P1, [256,256+d) O0, [256+d,256+2d) O1.
+// Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA raises a flag in shared
+// memory, writes the device status word, lets every role drain, frees TMEM and returns.
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace mka {
-bool fwd_tc_eligible(const FwdParams&, int) { return false; }
-cudaError_t launch_fwd_tc(const FwdParams&, unsigned int*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kNumQ = 2;
+constexpr int kThreads = 320;
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr uint32_t kPanelBytes = 128 * 128;          // [128 rows][64 bf16] with 128-byte rows
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+constexpr float kRescaleThreshold = 8.0f;            // log2 units
+
+struct TcMaps {
+    CUtensorMap q;
+    CUtensorMap k[3];
+    CUtensorMap v[3];
+};
+
+struct TcParams {
+    __nv_bfloat16* O;
+    float* LSE;
+    const float* gate;
+    long long n[3];
+    int B, H, T;
+    int window, q_offset;
+    float scale_log2;
+    unsigned int* status;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long gtimer() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false when the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(b, parity)) return true;
+    const unsigned long long t0 = gtimer();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try(b, parity)) return true;
+        if (*abort_flag) return false;
+        if (gtimer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int x, int y, int z, int w, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)) : "memory");
+}
+// Shared-memory matrix descriptors (128-byte swizzle; 8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t panel_stride_bytes) {
+    return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((panel_stride_bytes >> 4) & 0x3FFF) << 16) | (64ull << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+                   "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+                   "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+                   "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+                   "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+                   "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+                   "r"(r[30]), "r"(r[31]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <int DH>
+struct Cfg {
+    static constexpr int kPanels = DH / 64;
+    static constexpr uint32_t kTileBytes = kPanels * kPanelBytes;
+    static constexpr int kStages = DH == 128 ? 2 : 4;
+    static constexpr uint32_t kSmemBytes = (kNumQ + 2 * kStages) * kTileBytes + 1024;
+    static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+};
+
+struct Barriers {
+    uint64_t q_full;
+    uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
+    uint64_t s_full[kNumQ], p_full[kNumQ], pv_done[kNumQ];
+};
+
+// Key-tile range [first, end) of a block of query rows [r0, r1] (inclusive) on one level.
+__device__ __forceinline__ void tile_range(int level, long long r0, long long r1, int q_offset, int window, long long n,
+                                           int& first, int& end) {
+    long long lo_f, hi_f, lo_l, hi_l;
+    visible_range(level, r0 + q_offset, window, n, 0, lo_f, hi_f);
+    visible_range(level, r1 + q_offset, window, n, 0, lo_l, hi_l);
+    const long long hi = hi_l > hi_f ? hi_l : hi_f;
+    if (hi <= lo_f) { first = end = 0; return; }
+    first = (int)(lo_f / kTileN);
+    end = (int)((hi + kTileN - 1) / kTileN);
+}
+
+template <int DH>
+__global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+    using C = Cfg<DH>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* sQ = smem;                                   // kNumQ tiles
+    uint8_t* sK = sQ + kNumQ * C::kTileBytes;             // kStages tiles
+    uint8_t* sV = sK + C::kStages * C::kTileBytes;        // kStages tiles
+    __shared__ Barriers bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.z, h = blockIdx.y;
+    const int qpair = gridDim.x - 1 - blockIdx.x;          // heaviest (latest) rows first
+    const long long m0 = (long long)qpair * (kNumQ * kTileM);
+    const long long m_last = (m0 + kNumQ * kTileM - 1 < p.T - 1) ? m0 + kNumQ * kTileM - 1 : p.T - 1;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(&bar.q_full, 1);
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(&bar.k_full[s], 1); mbar_init(&bar.k_empty[s], 1);
+            mbar_init(&bar.v_full[s], 1); mbar_init(&bar.v_empty[s], 1);
+        }
+        for (int q = 0; q < kNumQ; ++q) {
+            mbar_init(&bar.s_full[q], 1); mbar_init(&bar.p_full[q], kTileM); mbar_init(&bar.pv_done[q], 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    // the CTA's level-ordered key-tile list (same closed form in every role)
+    int first[3], end[3];
+#pragma unroll
+    for (int l = 0; l < 3; ++l) {
+        if (p.n[l] > 0) tile_range(l, m0, m_last, p.q_offset, p.window, p.n[l], first[l], end[l]);
+        else first[l] = end[l] = 0;
+    }
+    const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
+
+    if (warp == kProducerWarp) {
+        if (lane == 0) {
+            mbar_expect_tx(&bar.q_full, kNumQ * C::kTileBytes);
+#pragma unroll
+            for (int q = 0; q < kNumQ; ++q)
+#pragma unroll
+                for (int pn = 0; pn < C::kPanels; ++pn)
+                    tma_load_4d(sQ + q * C::kTileBytes + pn * kPanelBytes, &maps.q, pn * 64, (int)(m0 + q * kTileM), h, b, &bar.q_full);
+            int issued_k = 0, issued_v = 0;
+            bool ok = true;
+            for (int l = 0; l < 3 && ok; ++l) {
+                for (int kt = first[l]; kt < end[l]; ++kt) {
+                    const int e = issued_k;
+                    const int s = e % C::kStages;
+                    const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                    if (!mbar_wait(&bar.k_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
+                    mbar_expect_tx(&bar.k_full[s], C::kTileBytes);
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes, &maps.k[l], pn * 64, kt * kTileN, h, b, &bar.k_full[s]);
+                    ++issued_k;
+                    if (!mbar_wait(&bar.v_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
+                    mbar_expect_tx(&bar.v_full[s], C::kTileBytes);
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes, &maps.v[l], pn * 64, kt * kTileN, h, b, &bar.v_full[s]);
+                    ++issued_v;
+                }
+            }
+            // Before leaving, make sure every copy this lane issued has landed (bounded): the shared
+            // memory must not be handed to another CTA with a bulk copy still in flight.
+            mbar_wait(&bar.q_full, 0, abortp);
+            for (int i = issued_k > C::kStages ? issued_k - C::kStages : 0; i < issued_k; ++i)
+                mbar_wait(&bar.k_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+            for (int i = issued_v > C::kStages ? issued_v - C::kStages : 0; i < issued_v; ++i)
+                mbar_wait(&bar.v_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane == 0) {
+            bool ok = mbar_wait(&bar.q_full, 0, abortp);
+            tc_fence_after();
+            const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+            auto issue_qk = [&](int q, int s) {
+                const uint32_t qa = q_addr + q * C::kTileBytes, ka = k_addr + s * C::kTileBytes;
+#pragma unroll
+                for (int k = 0; k < DH / 16; ++k) {
+                    const uint32_t off = (k / 4) * kPanelBytes + (k % 4) * 32;
+                    mma_ss(tmem + q * kTileN, desc_kmajor(qa + off), desc_kmajor(ka + off), C::kIdescQK, k > 0);
+                }
+                mma_commit(&bar.s_full[q]);
+            };
+            auto issue_pv = [&](int q, int s, bool accumulate) {
+                const uint32_t va = v_addr + s * C::kTileBytes;
+#pragma unroll
+                for (int k = 0; k < kTileN / 16; ++k)
+                    mma_ts(tmem + 256 + q * DH, tmem + q * kTileN + k * 8, desc_mnmajor(va + k * 2048, kPanelBytes), C::kIdescPV,
+                           (accumulate || k > 0) ? 1u : 0u);
+                mma_commit(&bar.pv_done[q]);
+            };
+            for (int e = 0; e < E && ok; ++e) {
+                const int s = e % C::kStages;
+                const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                if (!mbar_wait(&bar.k_full[s], ph, abortp)) { ok = false; break; }
+                tc_fence_after();
+                issue_qk(0, s);
+                if (e > 0) {
+                    const int sp = (e - 1) % C::kStages;
+                    if (!mbar_wait(&bar.p_full[1], (uint32_t)(e - 1) & 1u, abortp)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_pv(1, sp, e - 1 > 0);
+                    mma_commit(&bar.v_empty[sp]);
+                }
+                issue_qk(1, s);
+                mma_commit(&bar.k_empty[s]);
+                if (!mbar_wait(&bar.v_full[s], ph, abortp)) { ok = false; break; }
+                if (!mbar_wait(&bar.p_full[0], (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                tc_fence_after();
+                issue_pv(0, s, e > 0);
+            }
+            if (ok && E > 0) {
+                const int sp = (E - 1) % C::kStages;
+                if (mbar_wait(&bar.p_full[1], (uint32_t)(E - 1) & 1u, abortp)) {
+                    tc_fence_after();
+                    issue_pv(1, sp, E - 1 > 0);
+                    mma_commit(&bar.v_empty[sp]);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warpgroups
+        const int q = warp >> 2;
+        const int row_in_tile = tid & (kTileM - 1);
+        const long long t = m0 + (long long)q * kTileM + row_in_tile;
+        const bool row_valid = t < p.T;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t s_addr = tmem + lane_base + q * kTileN;
+        const uint32_t o_addr = tmem + lane_base + 256 + q * DH;
+        const long long tq0 = m0 + (long long)q * kTileM;                      // first row of this query tile
+        const long long tq1 = (tq0 + kTileM - 1 < p.T - 1) ? tq0 + kTileM - 1 : p.T - 1;
+
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        int e = 0;
+        for (int l = 0; l < 3 && ok; ++l) {
+            if (first[l] == end[l]) continue;
+            float bias = -INFINITY;
+            long long lo = 0, hi = 0;
+            if (row_valid) {
+                const float g = p.gate[((long long)b * p.T + t) * 3 + l];
+                bias = g > 0.f ? log2f(g) : -INFINITY;
+                visible_range(l, t + p.q_offset, p.window, p.n[l], 0, lo, hi);
+            }
+            // key tiles visible to every row of THIS query tile need no element mask
+            int full_first = 0, full_end = 0;
+            if (tq0 <= tq1) {
+                long long lo_f, hi_f, lo_l, hi_l;
+                visible_range(l, tq0 + p.q_offset, p.window, p.n[l], 0, lo_f, hi_f);
+                visible_range(l, tq1 + p.q_offset, p.window, p.n[l], 0, lo_l, hi_l);
+                full_first = (int)((lo_l + kTileN - 1) / kTileN);
+                full_end = (int)(hi_f / kTileN);
+                if (tq1 - tq0 + 1 < kTileM) full_end = full_first;         // ragged query tile: always mask
+            }
+            for (int kt = first[l]; kt < end[l]; ++kt, ++e) {
+                ok = mbar_wait(&bar.s_full[q], (uint32_t)e & 1u, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                float s[kTileN];
+#pragma unroll
+                for (int c0 = 0; c0 < kTileN; c0 += 32) tmem_ld32(s_addr + c0, reinterpret_cast<uint32_t*>(s) + c0);
+                tmem_ld_wait();
+                const bool need_mask = !(kt >= full_first && kt < full_end);
+                if (need_mask) {
+                    const int c_lo = (int)max(-1LL, min(lo - (long long)kt * kTileN, (long long)kTileN));
+                    const int c_hi = (int)max(-1LL, min(hi - (long long)kt * kTileN, (long long)kTileN));
+#pragma unroll
+                    for (int c = 0; c < kTileN; ++c)
+                        if (c < c_lo || c >= c_hi) s[c] = -INFINITY;
+                }
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < kTileN; ++c) mx = fmaxf(mx, s[c]);
+                const float x_max = fmaf(mx, p.scale_log2, bias);            // -inf when the whole row is masked
+                const float m_new = fmaxf(m_run, x_max);
+                const bool grow = m_new > m_run + kRescaleThreshold;         // also true for the first finite max
+                const float m_use = grow ? m_new : m_run;
+                const float m_eff = m_use == -INFINITY ? 0.f : m_use;
+                const float alpha = grow ? (m_run == -INFINITY ? 0.f : ex2(m_run - m_use)) : 1.f;
+                const float shift = bias - m_eff;
+                float sum = 0.f;
+                uint32_t pk[kTileN / 2];
+#pragma unroll
+                for (int c = 0; c < kTileN; c += 2) {
+                    const float p0 = ex2(fmaf(s[c], p.scale_log2, shift));
+                    const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, shift));
+                    sum += p0 + p1;
+                    pk[c / 2] = pack_bf16(p0, p1);
+                }
+                l_run = fmaf(l_run, alpha, sum);
+                m_run = m_use;
+                tmem_st32(s_addr, pk);
+                tmem_st32(s_addr + 32, pk + 32);
+                // O accumulator rescale (only when some row of this warp moved its reference maximum)
+                if (e > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                    ok = mbar_wait(&bar.pv_done[q], (uint32_t)(e - 1) & 1u, abortp);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c0 = 0; c0 < DH; c0 += 32) {
+                        uint32_t o[32];
+                        tmem_ld32(o_addr + c0, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(o_addr + c0, o);
+                    }
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&bar.p_full[q]);
+            }
+        }
+        // ------------------------------------------------------------ epilogue
+        __nv_bfloat16* Orow = p.O + (((long long)b * p.H + h) * p.T + t) * DH;
+        if (ok && E > 0) {
+            ok = mbar_wait(&bar.pv_done[q], (uint32_t)(E - 1) & 1u, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+#pragma unroll
+            for (int c0 = 0; c0 < DH; c0 += 32) {
+                uint32_t o[32];
+                if (E > 0) {
+                    tmem_ld32(o_addr + c0, o);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = 0u;
+                }
+                if (row_valid) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 v;
+                        const float z = inv;   // rows with nothing visible: inv = 0 -> exact zeros
+                        v.x = pack_bf16(z > 0.f ? __uint_as_float(o[i]) * z : 0.f, z > 0.f ? __uint_as_float(o[i + 1]) * z : 0.f);
+                        v.y = pack_bf16(z > 0.f ? __uint_as_float(o[i + 2]) * z : 0.f, z > 0.f ? __uint_as_float(o[i + 3]) * z : 0.f);
+                        v.z = pack_bf16(z > 0.f ? __uint_as_float(o[i + 4]) * z : 0.f, z > 0.f ? __uint_as_float(o[i + 5]) * z : 0.f);
+                        v.w = pack_bf16(z > 0.f ? __uint_as_float(o[i + 6]) * z : 0.f, z > 0.f ? __uint_as_float(o[i + 7]) * z : 0.f);
+                        *reinterpret_cast<uint4*>(Orow + c0 + i) = v;
+                    }
+                }
+            }
+            if (row_valid && p.LSE)
+                p.LSE[((long long)b * p.H + h) * p.T + t] = l_run > 0.f ? (m_run + log2f(l_run)) * kLn2 : -INFINITY;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    }
+    return fn;
+}
+
+// [B, H, rows, d] bf16 tensor with element strides (sb, sh, sn, 1); box = 64 columns x 128 rows.
+bool make_map(CUtensorMap* map, const void* base, int d, long long rows, int H, int B, long long sn, long long sh, long long sb) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)H, (cuuint64_t)B};
+    // a dimension of extent 1 never uses its stride; give it a well-formed one
+    if (H == 1) sh = sn * rows;
+    if (B == 1) sb = sh * H;
+    cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+    cuuint32_t box[4] = {64, 128, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DH>
+cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_t st) {
+    TcMaps maps;
+    if (!make_map(&maps.q, fp.Q, DH, fp.T, fp.H, fp.B, DH, (long long)fp.T * DH, (long long)fp.H * fp.T * DH))
+        return cudaErrorNotSupported;
+    for (int l = 0; l < 3; ++l) {
+        if (fp.L[l].n == 0) { maps.k[l] = maps.q; maps.v[l] = maps.q; continue; }
+        if (!make_map(&maps.k[l], fp.L[l].k, DH, fp.L[l].n, fp.H, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb) ||
+            !make_map(&maps.v[l], fp.L[l].v, DH, fp.L[l].n, fp.H, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb))
+            return cudaErrorNotSupported;
+    }
+    TcParams p;
+    p.O = static_cast<__nv_bfloat16*>(fp.O);
+    p.LSE = fp.LSE;
+    p.gate = fp.gate;
+    for (int l = 0; l < 3; ++l) p.n[l] = fp.L[l].n;
+    p.B = fp.B; p.H = fp.H; p.T = fp.T;
+    p.window = fp.window; p.q_offset = fp.q_offset;
+    p.scale_log2 = fp.scale * kLog2e;
+    p.status = status_word;
+    cudaError_t e = cudaFuncSetAttribute(fwd_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<DH>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    dim3 grid((fp.T + kNumQ * kTileM - 1) / (kNumQ * kTileM), fp.H, fp.B);
+    fwd_tc_kernel<DH><<<grid, kThreads, Cfg<DH>::kSmemBytes, st>>>(maps, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool fwd_tc_eligible(const FwdParams& p, int dtype) {
+    if (dtype != MKA_BF16 || p.mode != MKA_MODE_FAST || p.decode) return false;
+    if (p.d != 64 && p.d != 128) return false;
+    if (p.H > 65535 || p.B > 65535) return false;
+    for (int l = 0; l < 3; ++l) {
+        const LevelDev& L = p.L[l];
+        if (L.n == 0) continue;
+        if (L.n > 0x7fffffffLL) return false;
+        if (L.sn % 8 || L.sn <= 0) return false;
+        if (p.H > 1 && (L.sh % 8 || L.sh <= 0)) return false;
+        if (p.B > 1 && (L.sb % 8 || L.sb <= 0)) return false;
+    }
+    return encode_fn() != nullptr;
+}
+
+cudaError_t launch_fwd_tc(const FwdParams& p, unsigned int* status_word, cudaStream_t st) {
+    if (p.B == 0 || p.H == 0 || p.T == 0) return cudaSuccess;
+    return p.d == 128 ? launch_t<128>(p, status_word, st) : launch_t<64>(p, status_word, st);
+}
+
+}  // namespace mka

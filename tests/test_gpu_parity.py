@@ -91,8 +91,11 @@ def test_fwd_fast_matches_oracle(mka, orc, case, dtype, flags):
     P = problem(11, B, H, T, d, N, 64, dtype, router_std=0.3)
     gate = mka.mka_router(P["X"], P["W_r"], None)
     shape = mka.make_shape(B, H, T, d, 64, W, q_off, dtype=_dt(mka, dtype), flags=flags)
-    O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
-    torch.cuda.synchronize()
+    # bf16 without the force flag must take the tensor-core kernel, everything else the CUDA-core one
+    assert mka.mka_fwd_kernel_kind(shape, P["K"], P["V"]) == (1 if (dtype == torch.bfloat16 and not flags) else 0)
+    ws = mka.alloc_workspace(shape, N, mka.binding.MKA_WS_FWD, "cuda")
+    O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate, ws=ws)
+    assert mka.mka_device_status(ws) == 0
     rg, _ = orc.router(np64(P["X"]), np64(P["W_r"]))
     Or, Lr = orc.fwd(P["Q"], P["K"], P["V"], rg, W, q_off)
     check(O, Or, dtype, "O")
