@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the FastMKA hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c5|c4] [--legs c4,c5]
+                    [--impl ours|reference] [--no-e2e] [--no-cpu-baseline]
+
+One JSON line on stdout (rank 0).  A "step" is one pass of the path over one batch of seeded synthetic
+input of the named configuration:
+    c2 / c3 (prefill)   mka_router -> mka_fwd
+    c5      (training)  mka_router -> mka_fwd -> mka_bwd
+    c4      (decode)    mka_router -> mka_decode
+The headline `value` is the primary workload's algorithmic throughput (visible query-key pairs only) with
+inputs resident in HBM; `legs` holds the same measurement for the other configurations, each with its own
+roofline entry.  `e2e` repeats the primary workload with pinned HOST buffers: host->device copies of every
+input and the device->host read of the result are inside the timed region.  `--impl reference` times the
+CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from mka_inputs import CONFIGS, make_tensor  # noqa: E402
+
+DATASHEET = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
+FALLBACK = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": float(d["bf16_tflops"]), "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return dict(FALLBACK, source="fallback")
+
+
+def algorithmic_work(cfg):
+    """Flops / bytes the method itself must do (visible pairs only)."""
+    pairs = cfg.visible_pairs_per_head() * cfg.B * cfg.H
+    return {"pairs": pairs, "fwd_flops": 4.0 * cfg.d * pairs, "bwd_flops": 10.0 * cfg.d * pairs,
+            "decode_bytes": 2.0 * 2.0 * cfg.d * sum(cfg.N) * cfg.B * cfg.H}
+
+
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------ ours
+class Leg:
+    """One configuration resident on the device plus the calls of its step."""
+
+    def __init__(self, name, device, seed_shift=0):
+        import paper_2603_20586_b200 as mka
+        self.mka, self.name, self.dev = mka, name, device
+        cfg = CONFIGS[name]
+        if seed_shift:
+            cfg = type(cfg)(**{**cfg.__dict__, "seed": cfg.seed + 1000 * seed_shift})
+        self.cfg = cfg
+        self.work = algorithmic_work(cfg)
+        names = ["X", "W_r", "Q", "K1", "V1", "K2", "V2", "K3", "V3"] + (["dO"] if name == "c5" else [])
+        self.t = {n: make_tensor(cfg, n, device) for n in names}
+        B, H, T, d, D = cfg.B, cfg.H, cfg.T, cfg.d, cfg.D
+        self.K = [self.t["K1"], self.t["K2"], self.t["K3"]]
+        self.V = [self.t["V1"], self.t["V2"], self.t["V3"]]
+        self.shape = mka.make_shape(B, H, T, d, D, cfg.W, 0)
+        self.gate = torch.empty(B, T, 3, device=device)
+        self.O = torch.empty_like(self.t["Q"])
+        self.LSE = torch.empty(B, H, T, device=device)
+        which = {"c4": mka.MKA_WS_DECODE, "c5": mka.MKA_WS_BWD}.get(name, mka.MKA_WS_FWD)
+        self.ws = mka.alloc_workspace(self.shape, cfg.N, which, device)
+        self.launches = 0
+        if name == "c4":
+            self.q = self.t["Q"].view(B, H, d)
+            self.Od = torch.empty_like(self.q)
+            self.gate_d = self.gate.view(B, 3)
+            self.LSEd = self.LSE.view(B, H)
+            self.launches_per_step = 1 + 2          # router, decode partial, decode combine
+        elif name == "c5":
+            self.grads = {"dQ": torch.empty_like(self.t["Q"]), "dK": [torch.empty_like(k) for k in self.K],
+                          "dV": [torch.empty_like(v) for v in self.V], "dG": torch.empty(B, T, 3, device=device),
+                          "dW_r": torch.empty(D, 3, device=device), "db_r": torch.empty(3, device=device)}
+            self.launches_per_step = 1 + 1 + (1 + 1 + 3 + 1) + 3   # router, fwd, bwd(delta,dq,3 dkv,dgate), router bwd
+        else:
+            self.launches_per_step = 2              # router, fwd
+        self.ev = []
+
+    def step(self, record=False):
+        mka, t = self.mka, self.t
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
+        if record:
+            e[0].record()
+        mka.mka_router(t["X"], t["W_r"], None, gate=self.gate)
+        if record:
+            e[1].record()
+        if self.name == "c4":
+            mka.mka_decode(self.shape, self.q, self.K, self.V, self.gate_d, O=self.Od, LSE=self.LSEd, ws=self.ws)
+        else:
+            mka.mka_fwd(self.shape, t["Q"], self.K, self.V, self.gate, O=self.O, LSE=self.LSE, ws=self.ws)
+        if record:
+            e[2].record()
+        if self.name == "c5":
+            g = self.grads
+            mka.mka_bwd(self.shape, t["Q"], self.K, self.V, self.gate, self.O, self.LSE, t["dO"], R=t["X"], dQ=g["dQ"],
+                        dK=g["dK"], dV=g["dV"], dG=g["dG"], dW_r=g["dW_r"], db_r=g["db_r"], ws=self.ws)
+        if record:
+            e[3].record()
+            self.ev.append(e)
+
+    def result_tensor(self):
+        return self.Od if self.name == "c4" else (self.grads["dQ"] if self.name == "c5" else self.O)
+
+    def kernel_ms(self):
+        """Average device time of (router, main kernel, backward) over the recorded steps."""
+        r = [statistics.mean(a[i].elapsed_time(a[i + 1]) for a in self.ev) for i in range(3)]
+        return {"router": r[0], "main": r[1], "bwd": r[2]}
+
+
+def timed_steps(leg, steps, warmup, dist=None):
+    for _ in range(warmup):
+        leg.step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    leg.ev = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        leg.step(record=True)
+    t1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1)
+    if dist is not None:
+        tt = torch.tensor([ms], device=leg.dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    if leg.mka.mka_device_status(leg.ws) != 0:
+        raise RuntimeError("device status word reports a timed-out wait")
+    return ms / steps
+
+
+def leg_report(leg, ms_per_step, n_gpus, peaks):
+    cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
+    if leg.name == "c4":
+        achieved = w["decode_bytes"] / (k["main"] * 1e-3) / 1e9
+        roof = {"kernel": "decode_partial_kernel+decode_combine_kernel", "bound": "hbm", "achieved": achieved,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "frac_datasheet": achieved / DATASHEET["hbm_gbs"], "peak_source": peaks["source"], "traffic": None}
+        value = n_gpus * w["decode_bytes"] / (ms_per_step * 1e-3) / 1e9
+        unit, metric = "GB/s", "decode_hbm_gbs"
+    else:
+        achieved = w["fwd_flops"] / (k["main"] * 1e-3) / 1e12
+        roof = {"kernel": "fwd_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                "frac_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                "frac_datasheet": achieved / DATASHEET["bf16_tflops"], "peak_source": peaks["source"], "traffic": None}
+        flops = w["fwd_flops"] + (w["bwd_flops"] if leg.name == "c5" else 0.0)
+        value = n_gpus * flops / (ms_per_step * 1e-3) / 1e12
+        unit, metric = "TFLOP/s", ("fwd_bwd_tflops" if leg.name == "c5" else "prefill_fwd_tflops")
+    rep = {"workload": leg.name, "metric": metric, "value": value, "unit": unit, "ms_per_step": ms_per_step,
+           "kernel_ms": k, "roofline": roof}
+    if leg.name == "c5":
+        rep["bwd_tflops"] = w["bwd_flops"] / (k["bwd"] * 1e-3) / 1e12
+    return rep
+
+
+def e2e_run(leg, steps, warmup):
+    """Same step with pinned host inputs: H2D of every input and D2H of the result inside the timed region."""
+    names = list(leg.t.keys())
+    host = {n: torch.empty(leg.t[n].shape, dtype=leg.t[n].dtype, pin_memory=True).copy_(leg.t[n]) for n in names}
+    res = leg.result_tensor()
+    host_out = torch.empty(res.shape, dtype=res.dtype, pin_memory=True)
+    h2d = sum(h.numel() * h.element_size() for h in host.values())
+    d2h = host_out.numel() * host_out.element_size()
+
+    def one():
+        for n in names:
+            leg.t[n].copy_(host[n], non_blocking=True)
+        leg.step()
+        host_out.copy_(leg.result_tensor(), non_blocking=True)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        one()
+    t1.record()
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / steps, h2d, d2h
+
+
+# ------------------------------------------------------------------------------------------------ oracle arm
+_ROUTER_INPUTS = {}
+
+
+def _router_inputs(cfg):
+    """Router input and weights of a configuration (generated once per process; not part of any timing)."""
+    if cfg.name not in _ROUTER_INPUTS:
+        _ROUTER_INPUTS[cfg.name] = (make_tensor(cfg, "X").double().numpy(), make_tensor(cfg, "W_r").double().numpy())
+    return _ROUTER_INPUTS[cfg.name]
+
+
+def oracle_sample(name, budget_rows=None):
+    """Times the CPU oracle, as it stands, on a bounded seeded sample of workload `name`."""
+    from oracle import mka_oracle as orc
+    orc.build()
+    cfg = CONFIGS[name]
+    rng = np.random.default_rng(1234 + cfg.seed)
+    cores = orc.num_threads()
+    d, W = cfg.d, cfg.W
+    if name == "c4":
+        heads = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(64)]
+        per = cfg.H * 1
+        X, Wr = _router_inputs(cfg)
+        gate, _ = orc.router(X, Wr)
+        dt = 0.0
+        for (b, h) in heads:
+            def sl(nm, n):
+                off = ((b * cfg.H + h) * n) * d
+                return make_tensor(cfg, nm, flat_start=off, flat_count=n * d).double().numpy().reshape(1, 1, n, d)
+            K = [sl(f"K{l + 1}", cfg.N[l]) for l in range(3)]
+            V = [sl(f"V{l + 1}", cfg.N[l]) for l in range(3)]
+            q = make_tensor(cfg, "Q", flat_start=(b * cfg.H + h) * d, flat_count=d).double().numpy().reshape(1, 1, 1, d)
+            t0 = time.perf_counter()
+            orc.fwd(q, K, V, gate[b:b + 1], 1, decode=True)
+            dt += time.perf_counter() - t0
+        bytes_ = 2.0 * 2.0 * d * sum(cfg.N) * len(heads)
+        return {"value": bytes_ / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle", "seconds": dt,
+                "sample": f"{len(heads)} of {cfg.B * cfg.H} (batch, head) pairs, all {sum(cfg.N)} cached rows each"}
+    # prefill / training: a few heads, a seeded sample of query rows
+    n_heads = 2
+    n_rows = budget_rows or (1024 if name == "c3" else 2048)
+    n_rows = min(n_rows, cfg.T)
+    heads = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(n_heads)]
+    rows = np.sort(rng.choice(cfg.T, size=n_rows, replace=False))
+    X, Wr = _router_inputs(cfg)
+    t_all, pairs = 0.0, 0
+    t0 = time.perf_counter()
+    gate, _ = orc.router(X, Wr)
+    t_all += time.perf_counter() - t0
+    for (b, h) in heads:
+        def sl(nm, n):
+            off = ((b * cfg.H + h) * n) * d
+            return make_tensor(cfg, nm, flat_start=off, flat_count=n * d).double().numpy().reshape(1, 1, n, d)
+        Q = sl("Q", cfg.T)
+        K = [sl(f"K{l + 1}", cfg.N[l]) for l in range(3)]
+        V = [sl(f"V{l + 1}", cfg.N[l]) for l in range(3)]
+        t0 = time.perf_counter()
+        orc.fwd(Q, K, V, gate[b:b + 1], W, rows=rows)
+        if name == "c5":
+            dO = sl("dO", cfg.T)
+            orc.bwd(Q, K, V, gate[b:b + 1], dO, W, rows=rows, want_kv=False)
+        t_all += time.perf_counter() - t0
+        for t in rows:
+            pairs += min(t + 1, W) + (t + 1) + cfg.N[2]
+    flops = (4.0 if name != "c5" else 14.0) * d * pairs
+    return {"value": flops / t_all / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "seconds": t_all,
+            "sample": f"{n_heads} (batch, head) pairs x {n_rows} seeded query rows of {cfg.T}"
+                      + (" (forward + dQ/dG backward rows)" if name == "c5" else "") + "; router on all tokens"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5"])
+    ap.add_argument("--legs", default="c4,c5,c2", help="other configurations measured after the primary one ('' = none)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = CONFIGS[args.workload]
+    metric_name = "decode_hbm_gbs" if args.workload == "c4" else ("fwd_bwd_tflops" if args.workload == "c5" else "prefill_fwd_tflops")
+    base = {"metric": f"FastMKA {metric_name} (algorithmic, visible pairs only)", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
+            "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+            "config": {"workload": f"{args.workload}: B={cfg.B} H={cfg.H} d={cfg.d} D={cfg.D} T={cfg.T} W={cfg.W} N={list(cfg.N)} seed={cfg.seed}",
+                       "l2": "inputs larger than L2 (no flush needed)" if args.workload != "c2" else "inputs ~235 MB, larger than the 126 MB L2",
+                       "per_gpu": "each rank runs the whole configuration on its own seeded batch (no collective on the data path)"}}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        vals = []
+        for _ in range(args.warmup):
+            oracle_sample(args.workload, budget_rows=64)
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            vals.append(oracle_sample(args.workload, budget_rows=256 if args.workload != "c4" else None))
+        dt = (time.perf_counter() - t0) / max(1, args.steps)
+        v = statistics.mean(x["value"] for x in vals)
+        cb = dict(vals[-1], value=v)
+        out = dict(base, impl="reference", value=v, unit=cb["unit"], ms_per_step=dt * 1e3, dtype="f64", cpu_baseline=cb,
+                   e2e={"value": v, "unit": cb["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, gpu_launches=0,
+                   n_gpus=args.gpus)
+        print(json.dumps(out))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    peaks = load_peaks()
+    sampler = ClockSampler(local)
+    leg = Leg(args.workload, dev, seed_shift=rank)
+    sampler.start()
+    ms = timed_steps(leg, args.steps, args.warmup, dist)
+    clocks = sampler.stop()
+    rep = leg_report(leg, ms, world, peaks)
+    launches = leg.launches_per_step * args.steps
+    out = dict(base, value=rep["value"], unit=rep["unit"], ms_per_step=ms, roofline=rep["roofline"], kernel_ms=rep["kernel_ms"],
+               clocks=clocks, gpu_launches=launches, n_gpus=world)
+    if "bwd_tflops" in rep:
+        out["bwd_tflops"] = rep["bwd_tflops"]
+    if not args.no_e2e:
+        e_ms, h2d, d2h = e2e_run(leg, max(2, min(args.steps, 5)), 1)
+        w = leg.work
+        if args.workload == "c4":
+            ev = world * w["decode_bytes"] / (e_ms * 1e-3) / 1e9
+        else:
+            ev = world * (w["fwd_flops"] + (w["bwd_flops"] if args.workload == "c5" else 0.0)) / (e_ms * 1e-3) / 1e12
+        out["e2e"] = {"value": ev, "unit": rep["unit"], "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    del leg
+    torch.cuda.empty_cache()
+    legs = []
+    if world == 1:
+        for name in [x for x in args.legs.split(",") if x and x != args.workload]:
+            l2 = Leg(name, dev)
+            k = max(3, min(args.steps, 5)) if name != "c4" else max(3, min(args.steps, 10))
+            ms2 = timed_steps(l2, k, 3)
+            legs.append(leg_report(l2, ms2, 1, peaks))
+            del l2
+            torch.cuda.empty_cache()
+    out["legs"] = legs
+    if rank == 0:
+        if not args.no_cpu_baseline and world == 1:
+            out["cpu_baseline"] = oracle_sample(args.workload)
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

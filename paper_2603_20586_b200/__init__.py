@@ -1,8 +1,25 @@
 """B200 (sm_100a) FastMKA attention library: Python binding of the C ABI in ``include/mka.h``.
 
-The package holds the CUDA sources (``csrc/``), the build step (``build.py``) and the ctypes binding.
-Importing it requires the built library; there is no CPU or PyTorch fallback.
+The package holds the CUDA sources (``csrc/``), the build step (``build.py``) and the ctypes binding
+(``binding.py``).  Attributes are resolved lazily from the binding so that
+``python -m paper_2603_20586_b200.build`` can run before the library exists; the first use of any
+entry point loads ``libmka_b200.so`` and raises if it is missing or stale.  There is no CPU or
+PyTorch fallback.
 """
-from .binding import *  # noqa: F401,F403
-from .binding import (MkaError, lib, make_shape, mka_bwd, mka_decode, mka_decode_plan, mka_device_status,  # noqa: F401
-                      mka_fwd, mka_fwd_kernel_kind, mka_fwd_tile_range, mka_router, mka_workspace_bytes, alloc_workspace, status_str)
+import importlib
+
+_BINDING = None
+
+
+def __getattr__(name):
+    global _BINDING
+    if name == "build":
+        return importlib.import_module(".build", __name__)
+    if _BINDING is None:
+        _BINDING = importlib.import_module(".binding", __name__)
+    if name == "binding":
+        return _BINDING
+    try:
+        return getattr(_BINDING, name)
+    except AttributeError:
+        raise AttributeError(f"module {__name__!r} has no attribute {name!r}") from None
