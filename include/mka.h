@@ -171,6 +171,31 @@ mka_status mka_bwd(const mka_shape* shape, const void* Q, const mka_level L[3], 
                    void* dQ, const mka_level_grad dL[3], float* dG, float* dW_r, float* db_r,
                    void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * Decode for callers that cannot provide scratch memory (the paper has no counterpart; this entry
+ * point exists for deployment reasons only).  Same computation, arguments and results as mka_decode,
+ * but without `ws`: the per-chunk partials are kept in an 8 MiB array that is compiled into the
+ * library, so the call performs no device allocation of any kind and needs none from its caller.
+ * It is meant for hosts where allocating is not an option at call time: serving engines that claim
+ * all device memory for their own pool at start-up (a later cudaMalloc there fails or has to wait for
+ * the device to go idle), latency-bound decode loops that may not stall on the allocator's implicit
+ * device synchronisation, and plug-ins that only ever receive raw input/output pointers from a
+ * runtime whose memory plan is fixed before the first token.
+ *   - Limit: B * H * total_chunks * (d + 2) floats (total_chunks from mka_decode_plan) must fit in
+ *     mka_decode_static_max_bytes() = 8 MiB; larger problems are rejected with MKA_ERR_WORKSPACE and
+ *     nothing is launched.  (For d = 128 that is 16131 chunk partials, e.g. 32 heads x 516k cached rows.)
+ *   - The array costs 8 MiB on every GPU that loads the library, for the life of the process.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and remembers it; make that first call during set-up, before any stream capture begins.
+ *   - All calls on one device share the one array and it keeps whatever the last call wrote.  Nothing
+ *     in it needs clearing between calls (every slot that is read was written by the same call), but
+ *     two calls whose kernels overlap on the GPU -- different streams, no ordering between them --
+ *     race on it and produce garbage.  Serialise such calls or use mka_decode with separate workspaces.
+ */
+mka_status mka_decode_static(const mka_shape* shape, const void* q, const mka_level L[3], const float* gate,
+                             void* O, float* LSE, void* stream);
+size_t mka_decode_static_max_bytes(void);
+
 /* Integer bookkeeping, exposed so that it can be checked bit for bit (host functions, no CUDA call). */
 mka_status mka_decode_plan(const int64_t n_level[3], int32_t B, int32_t H, int32_t d, mka_decode_plan_t* plan);
 mka_status mka_fwd_tile_range(const mka_shape* shape, const int64_t n_level[3], int32_t level,

@@ -23,7 +23,8 @@ MKA_WS_FWD, MKA_WS_DECODE, MKA_WS_BWD = 0, 1, 2
 TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
-           "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind"]
+           "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
+           "mka_decode_static", "mka_decode_static_max_bytes"]
 
 
 class MkaError(RuntimeError):
@@ -77,9 +78,12 @@ def _load() -> ctypes.CDLL:
     lib.mka_fwd_tile_range.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(ctypes.c_int64), i32, i64,
                                        ctypes.POINTER(mka_tile_range)]
     lib.mka_device_status.argtypes = [vp, vp]
+    lib.mka_decode_static.argtypes = [ctypes.POINTER(mka_shape), vp, ctypes.POINTER(mka_level), vp, vp, vp, vp]
+    lib.mka_decode_static_max_bytes.restype = ctypes.c_size_t
+    lib.mka_decode_static_max_bytes.argtypes = []
     lib.mka_fwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level)]
     for name in EXPORTS:
-        if name not in ("mka_status_str", "mka_workspace_bytes"):
+        if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes"):
             getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -196,6 +200,20 @@ def mka_decode(shape: mka_shape, q, K, V, gate, O=None, LSE=None, ws=None, strea
     _check(lib.mka_decode(ctypes.byref(shape), _ptr(q), _levels(K, V), _ptr(gate), _ptr(O), _ptr(LSE), _ptr(ws),
                           ws.numel(), _stream(stream)), "mka_decode")
     return O, LSE
+
+
+def mka_decode_static(shape: mka_shape, q, K, V, gate, O, LSE=None, stream=None):
+    """Decode without a workspace, for callers that may not allocate: the partials go to the 8 MiB array
+    built into the library.  This wrapper allocates nothing either -- `O` (and `LSE`, if wanted) must be
+    passed in.  Raises MkaError(4) when the problem's split table does not fit the built-in array."""
+    assert q.is_contiguous() and gate.is_contiguous() and gate.dtype == torch.float32 and O.is_contiguous()
+    _check(lib.mka_decode_static(ctypes.byref(shape), _ptr(q), _levels(K, V), _ptr(gate), _ptr(O), _ptr(LSE),
+                                 _stream(stream)), "mka_decode_static")
+    return O, LSE
+
+
+def mka_decode_static_max_bytes() -> int:
+    return int(lib.mka_decode_static_max_bytes())
 
 
 def mka_bwd(shape: mka_shape, Q, K, V, gate, O, LSE, dO, R=None, dQ=None, dK=None, dV=None, dG=None, dW_r=None,

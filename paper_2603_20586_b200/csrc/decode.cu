@@ -7,6 +7,8 @@
 // warp shuffles / shared memory into one UN-GATED partial per chunk: (m_c, z_c, acc_c[d]).
 // Kernel 2: per (batch, head), gate-weighted log-sum-exp combine over all chunks of all levels:
 //   O = sum_c lam_{l(c)} 2^{m_c-M} acc_c / sum_c lam_{l(c)} 2^{m_c-M} z_c.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mka {
@@ -216,3 +218,91 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st) {
 }
 
 }  // namespace mka
+
+// ---------------------------------------------------------------------------------------------
+// mka_decode_static: the decode entry point for callers that cannot hand over scratch memory.
+// The per-chunk partials live in the file-scope device array below instead of a caller workspace.
+// Every GPU that loads this library carries the array (8 MiB) until the process exits.
+namespace mka {
+namespace {
+
+constexpr size_t kStaticScratchFloats = (size_t)2 << 20;                    // 2 Mi floats = 8 MiB
+static __device__ __align__(256) float g_decode_static_scratch[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_ptr[kMaxDevices];       // device address of the array, per device ordinal
+std::mutex g_static_scratch_mutex;
+
+// In host code the array's name is only a handle; the address a kernel can use has to be asked for,
+// once per device and with that device current.
+cudaError_t static_scratch_address(float** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_ptr[dev]) {
+        float* ptr = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_decode_static_scratch);
+        if (e != cudaSuccess) return e;
+        if (!ptr) return cudaErrorInvalidSymbol;
+        g_static_scratch_ptr[dev] = ptr;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return cudaSuccess;
+}
+
+inline bool is_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+}  // namespace mka
+
+extern "C" size_t mka_decode_static_max_bytes(void) { return mka::kStaticScratchFloats * sizeof(float); }
+
+extern "C" mka_status mka_decode_static(const mka_shape* s, const void* q, const mka_level L[3], const float* gate,
+                                        void* O, float* LSE, void* stream) {
+    using namespace mka;
+    if (!s || !L) return MKA_ERR_ARG;
+    if (s->dtype != MKA_BF16 || s->mode != MKA_MODE_FAST) return MKA_ERR_UNSUPPORTED;
+    if (s->B < 0 || s->H < 0 || s->T != 1) return MKA_ERR_SHAPE;
+    if (s->d != 64 && s->d != 128) return MKA_ERR_SHAPE;
+    int64_t n_level[3];
+    for (int l = 0; l < 3; ++l) {
+        n_level[l] = L[l].n;
+        if (L[l].n < 0) return MKA_ERR_SHAPE;
+        if (L[l].n == 0) continue;
+        if (!L[l].k || !L[l].v) return MKA_ERR_ARG;
+        if (L[l].stride_n < s->d || L[l].stride_b < 0 || L[l].stride_h < 0) return MKA_ERR_SHAPE;
+        if (!is_aligned16(L[l].k) || !is_aligned16(L[l].v)) return MKA_ERR_ALIGN;
+        if (L[l].stride_n % 8 || L[l].stride_b % 8 || L[l].stride_h % 8) return MKA_ERR_ALIGN;
+    }
+    if (s->B == 0 || s->H == 0) return MKA_OK;
+    if (!q || !gate || !O) return MKA_ERR_ARG;
+    if (!is_aligned16(q) || !is_aligned16(O)) return MKA_ERR_ALIGN;
+    mka_decode_plan_t plan;
+    mka_status st = mka_decode_plan(n_level, s->B, s->H, s->d, &plan);
+    if (st != MKA_OK) return st;
+    const unsigned long long slots = (unsigned long long)s->B * s->H * (unsigned long long)plan.total_chunks;
+    if (slots > 0x7fffffffULL) return MKA_ERR_SHAPE;
+    // the split table of this problem needs more partial slots than the built-in array holds
+    if (slots * (unsigned long long)(s->d + 2) > kStaticScratchFloats) return MKA_ERR_WORKSPACE;
+    float* scratch = nullptr;
+    if (static_scratch_address(&scratch) != cudaSuccess) return MKA_ERR_CUDA;
+    DecodeParams p;
+    p.q = q; p.O = O; p.LSE = LSE; p.gate = gate;
+    for (int l = 0; l < 3; ++l) {
+        p.L[l].k = L[l].k; p.L[l].v = L[l].v; p.L[l].n = L[l].n;
+        p.L[l].sb = L[l].stride_b; p.L[l].sh = L[l].stride_h; p.L[l].sn = L[l].stride_n;
+        p.n_chunks[l] = plan.n_chunks[l];
+    }
+    p.B = s->B; p.H = s->H; p.d = s->d;
+    p.scale = s->scale > 0.f ? s->scale : 1.0f / sqrtf((float)s->d);
+    p.chunk_rows = plan.chunk_rows;
+    p.total_chunks = plan.total_chunks;
+    // Nothing in the array has to start at zero: the partial kernel writes every slot that the combine
+    // kernel of the same call reads, so whatever an earlier call left behind is never looked at.
+    p.partial = scratch;
+    cudaError_t e = launch_decode(p, static_cast<cudaStream_t>(stream));
+    if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
