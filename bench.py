@@ -65,7 +65,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -110,7 +110,8 @@ class Leg:
             cfg = type(cfg)(**{**cfg.__dict__, "seed": cfg.seed + 1000 * seed_shift})
         self.cfg = cfg
         self.work = algorithmic_work(cfg)
-        names = ["X", "W_r", "Q", "K1", "V1", "K2", "V2", "K3", "V3"] + (["dO"] if name == "c5" else [])
+        self.kind = {"c4": "decode", "c5": "train"}.get(name[:2], "prefill")
+        names = ["X", "W_r", "Q", "K1", "V1", "K2", "V2", "K3", "V3"] + (["dO"] if self.kind == "train" else [])
         self.t = {n: make_tensor(cfg, n, device) for n in names}
         B, H, T, d, D = cfg.B, cfg.H, cfg.T, cfg.d, cfg.D
         self.K = [self.t["K1"], self.t["K2"], self.t["K3"]]
@@ -119,16 +120,16 @@ class Leg:
         self.gate = torch.empty(B, T, 3, device=device)
         self.O = torch.empty_like(self.t["Q"])
         self.LSE = torch.empty(B, H, T, device=device)
-        which = {"c4": mka.MKA_WS_DECODE, "c5": mka.MKA_WS_BWD}.get(name, mka.MKA_WS_FWD)
+        which = {"decode": mka.MKA_WS_DECODE, "train": mka.MKA_WS_BWD}.get(self.kind, mka.MKA_WS_FWD)
         self.ws = mka.alloc_workspace(self.shape, cfg.N, which, device)
         self.launches = 0
-        if name == "c4":
+        if self.kind == "decode":
             self.q = self.t["Q"].view(B, H, d)
             self.Od = torch.empty_like(self.q)
             self.gate_d = self.gate.view(B, 3)
             self.LSEd = self.LSE.view(B, H)
             self.launches_per_step = 1 + 2          # router, decode partial, decode combine
-        elif name == "c5":
+        elif self.kind == "train":
             self.grads = {"dQ": torch.empty_like(self.t["Q"]), "dK": [torch.empty_like(k) for k in self.K],
                           "dV": [torch.empty_like(v) for v in self.V], "dG": torch.empty(B, T, 3, device=device),
                           "dW_r": torch.empty(D, 3, device=device), "db_r": torch.empty(3, device=device)}
@@ -145,13 +146,13 @@ class Leg:
         mka.mka_router(t["X"], t["W_r"], None, gate=self.gate)
         if record:
             e[1].record()
-        if self.name == "c4":
+        if self.kind == "decode":
             mka.mka_decode(self.shape, self.q, self.K, self.V, self.gate_d, O=self.Od, LSE=self.LSEd, ws=self.ws)
         else:
             mka.mka_fwd(self.shape, t["Q"], self.K, self.V, self.gate, O=self.O, LSE=self.LSE, ws=self.ws)
         if record:
             e[2].record()
-        if self.name == "c5":
+        if self.kind == "train":
             g = self.grads
             mka.mka_bwd(self.shape, t["Q"], self.K, self.V, self.gate, self.O, self.LSE, t["dO"], R=t["X"], dQ=g["dQ"],
                         dK=g["dK"], dV=g["dV"], dG=g["dG"], dW_r=g["dW_r"], db_r=g["db_r"], ws=self.ws)
@@ -160,7 +161,7 @@ class Leg:
             self.ev.append(e)
 
     def result_tensor(self):
-        return self.Od if self.name == "c4" else (self.grads["dQ"] if self.name == "c5" else self.O)
+        return self.Od if self.kind == "decode" else (self.grads["dQ"] if self.kind == "train" else self.O)
 
     def kernel_ms(self):
         """Average device time of (router, main kernel, backward) over the recorded steps."""
@@ -197,7 +198,7 @@ def timed_steps(leg, steps, warmup, dist=None):
 
 def leg_report(leg, ms_per_step, n_gpus, peaks):
     cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
-    if leg.name == "c4":
+    if leg.kind == "decode":
         achieved = w["decode_bytes"] / (k["main"] * 1e-3) / 1e9
         roof = {"kernel": "decode_partial_kernel+decode_combine_kernel", "bound": "hbm", "achieved": achieved,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
@@ -210,12 +211,12 @@ def leg_report(leg, ms_per_step, n_gpus, peaks):
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                 "frac_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
                 "frac_datasheet": achieved / DATASHEET["bf16_tflops"], "peak_source": peaks["source"], "traffic": None}
-        flops = w["fwd_flops"] + (w["bwd_flops"] if leg.name == "c5" else 0.0)
+        flops = w["fwd_flops"] + (w["bwd_flops"] if leg.kind == "train" else 0.0)
         value = n_gpus * flops / (ms_per_step * 1e-3) / 1e12
-        unit, metric = "TFLOP/s", ("fwd_bwd_tflops" if leg.name == "c5" else "prefill_fwd_tflops")
+        unit, metric = "TFLOP/s", ("fwd_bwd_tflops" if leg.kind == "train" else "prefill_fwd_tflops")
     rep = {"workload": leg.name, "metric": metric, "value": value, "unit": unit, "ms_per_step": ms_per_step,
            "kernel_ms": k, "roofline": roof}
-    if leg.name == "c5":
+    if leg.kind == "train":
         rep["bwd_tflops"] = w["bwd_flops"] / (k["bwd"] * 1e-3) / 1e12
     return rep
 
@@ -266,7 +267,7 @@ def oracle_sample(name, budget_rows=None):
     rng = np.random.default_rng(1234 + cfg.seed)
     cores = orc.num_threads()
     d, W = cfg.d, cfg.W
-    if name == "c4":
+    if name[:2] == "c4":
         heads = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(64)]
         per = cfg.H * 1
         X, Wr = _router_inputs(cfg)
@@ -305,24 +306,24 @@ def oracle_sample(name, budget_rows=None):
         V = [sl(f"V{l + 1}", cfg.N[l]) for l in range(3)]
         t0 = time.perf_counter()
         orc.fwd(Q, K, V, gate[b:b + 1], W, rows=rows)
-        if name == "c5":
+        if name[:2] == "c5":
             dO = sl("dO", cfg.T)
             orc.bwd(Q, K, V, gate[b:b + 1], dO, W, rows=rows, want_kv=False)
         t_all += time.perf_counter() - t0
         for t in rows:
             pairs += min(t + 1, W) + (t + 1) + cfg.N[2]
-    flops = (4.0 if name != "c5" else 14.0) * d * pairs
+    flops = (4.0 if name[:2] != "c5" else 14.0) * d * pairs
     return {"value": flops / t_all / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "seconds": t_all,
             "sample": f"{n_heads} (batch, head) pairs x {n_rows} seeded query rows of {cfg.T}"
-                      + (" (forward + dQ/dG backward rows)" if name == "c5" else "") + "; router on all tokens"}
+                      + (" (forward + dQ/dG backward rows)" if name[:2] == "c5" else "") + "; router on all tokens"}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "c3p", "c4p", "c5p"])
     ap.add_argument("--legs", default="c4,c5,c2", help="other configurations measured after the primary one ('' = none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
@@ -332,7 +333,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     cfg = CONFIGS[args.workload]
-    metric_name = "decode_hbm_gbs" if args.workload == "c4" else ("fwd_bwd_tflops" if args.workload == "c5" else "prefill_fwd_tflops")
+    wk = args.workload[:2]
+    metric_name = "decode_hbm_gbs" if wk == "c4" else ("fwd_bwd_tflops" if wk == "c5" else "prefill_fwd_tflops")
     base = {"metric": f"FastMKA {metric_name} (algorithmic, visible pairs only)", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
             "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
@@ -348,7 +350,7 @@ def main():
             oracle_sample(args.workload, budget_rows=64)
         t0 = time.perf_counter()
         for _ in range(args.steps):
-            vals.append(oracle_sample(args.workload, budget_rows=256 if args.workload != "c4" else None))
+            vals.append(oracle_sample(args.workload, budget_rows=256 if wk != "c4" else None))
         dt = (time.perf_counter() - t0) / max(1, args.steps)
         v = statistics.mean(x["value"] for x in vals)
         cb = dict(vals[-1], value=v)
@@ -382,10 +384,10 @@ def main():
     if not args.no_e2e:
         e_ms, h2d, d2h = e2e_run(leg, max(2, min(args.steps, 5)), 1)
         w = leg.work
-        if args.workload == "c4":
+        if wk == "c4":
             ev = world * w["decode_bytes"] / (e_ms * 1e-3) / 1e9
         else:
-            ev = world * (w["fwd_flops"] + (w["bwd_flops"] if args.workload == "c5" else 0.0)) / (e_ms * 1e-3) / 1e12
+            ev = world * (w["fwd_flops"] + (w["bwd_flops"] if wk == "c5" else 0.0)) / (e_ms * 1e-3) / 1e12
         out["e2e"] = {"value": ev, "unit": rep["unit"], "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
     del leg
     torch.cuda.empty_cache()
@@ -393,7 +395,7 @@ def main():
     if world == 1:
         for name in [x for x in args.legs.split(",") if x and x != args.workload]:
             l2 = Leg(name, dev)
-            k = max(3, min(args.steps, 5)) if name != "c4" else max(3, min(args.steps, 10))
+            k = max(3, min(args.steps, 5)) if name != "c4" else max(3, min(args.steps, 20))
             ms2 = timed_steps(l2, k, 3)
             legs.append(leg_report(l2, ms2, 1, peaks))
             del l2
