@@ -133,7 +133,7 @@ class Leg:
             self.grads = {"dQ": torch.empty_like(self.t["Q"]), "dK": [torch.empty_like(k) for k in self.K],
                           "dV": [torch.empty_like(v) for v in self.V], "dG": torch.empty(B, T, 3, device=device),
                           "dW_r": torch.empty(D, 3, device=device), "db_r": torch.empty(3, device=device)}
-            self.launches_per_step = 1 + 1 + (1 + 1 + 3 + 1) + 3   # router, fwd, bwd(delta,dq,3 dkv,dgate), router bwd
+            self.launches_per_step = 1 + 1 + (1 + 1 + 1 + 1) + 3   # router, fwd, bwd(prep,dq,dkv,dgate), router bwd
         else:
             self.launches_per_step = 2              # router, fwd
         self.ev = []

@@ -165,6 +165,9 @@ mka_status mka_decode(const mka_shape* shape, const void* q, const mka_level L[3
  *   O, LSE: outputs of mka_fwd;  dO [B,H,T,d];  R [B*T, D] router input in r_dtype (NULL skips dW_r, db_r)
  *   dQ [B,H,T,d];  dL[3] gradient destinations (a level with n == 0 is skipped);  dG [B,T,3] f32;
  *   dW_r [D,3] f32 or NULL;  db_r [3] f32 or NULL.
+ * bf16 with d in {64,128} runs the TMA + tcgen05 kernels (one pass that owns query tiles for dQ and dG, one
+ * pass that owns key tiles for dK and dV; scores are recomputed in each, nothing is accumulated atomically);
+ * f32, other head widths and MKA_FLAG_FORCE_SIMT run the CUDA-core kernels.  Both are deterministic.
  */
 mka_status mka_bwd(const mka_shape* shape, const void* Q, const mka_level L[3], const float* gate,
                    const void* O, const float* LSE, const void* dO, const void* R, int32_t r_dtype,
@@ -204,6 +207,11 @@ mka_status mka_fwd_tile_range(const mka_shape* shape, const int64_t n_level[3], 
 /* Which forward kernel mka_fwd would run for this problem (host function, no launch):
  * 0 = CUDA-core kernel, 1 = TMA + tcgen05 tensor-core kernel, negative = arguments invalid. */
 int32_t mka_fwd_kernel_kind(const mka_shape* shape, const mka_level L[3]);
+
+/* Which kernels mka_bwd would run for this problem (host function, no launch): 0 = CUDA-core kernels,
+ * 1 = TMA + tcgen05 tensor-core kernels (bf16, d in {64,128}, 16-byte aligned strides), negative = arguments
+ * invalid.  dL may be NULL (then only the level sources decide). */
+int32_t mka_bwd_kernel_kind(const mka_shape* shape, const mka_level L[3], const mka_level_grad dL[3]);
 
 /* Synchronises `stream` and returns the device status word that the kernels of the last call using
  * `ws` left there: MKA_OK, or MKA_ERR_TIMEOUT when a bounded wait inside a kernel gave up (the

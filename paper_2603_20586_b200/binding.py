@@ -24,7 +24,7 @@ TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
-           "mka_decode_static", "mka_decode_static_max_bytes"]
+           "mka_bwd_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes"]
 
 
 class MkaError(RuntimeError):
@@ -82,6 +82,7 @@ def _load() -> ctypes.CDLL:
     lib.mka_decode_static_max_bytes.restype = ctypes.c_size_t
     lib.mka_decode_static_max_bytes.argtypes = []
     lib.mka_fwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level)]
+    lib.mka_bwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level), vp]
     for name in EXPORTS:
         if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes"):
             getattr(lib, name).restype = ctypes.c_int
@@ -254,6 +255,11 @@ def mka_bwd(shape: mka_shape, Q, K, V, gate, O, LSE, dO, R=None, dQ=None, dK=Non
 
 def mka_fwd_kernel_kind(shape: mka_shape, K, V) -> int:
     return int(lib.mka_fwd_kernel_kind(ctypes.byref(shape), _levels(K, V)))
+
+
+def mka_bwd_kernel_kind(shape: mka_shape, K, V) -> int:
+    """1 when mka_bwd would run the tensor-core kernels for this problem (gradients laid out like K, V)."""
+    return int(lib.mka_bwd_kernel_kind(ctypes.byref(shape), _levels(K, V), None))
 
 
 def mka_device_status(ws: torch.Tensor, stream=None) -> int:

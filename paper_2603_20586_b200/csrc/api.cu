@@ -50,6 +50,12 @@ void fill_levels(LevelDev out[3], const mka_level L[3]) {
 
 constexpr int kRouterBwdChunks = 128;
 
+// Per-row statistics of the tensor-core backward: three arrays of [B, H, Tpad] float2, Tpad = T rounded up to 64.
+size_t bwd_stats_bytes(const mka_shape* s) {
+    const size_t tpad = ((size_t)s->T + 63) / 64 * 64;
+    return (size_t)3 * s->B * s->H * tpad * 2 * sizeof(float);
+}
+
 }  // namespace
 
 extern "C" {
@@ -130,7 +136,8 @@ size_t mka_workspace_bytes(const mka_shape* s, const int64_t n_level[3], int32_t
     if (which == MKA_WS_BWD) {
         size_t rows = (size_t)s->B * s->H * s->T;
         return kWsHeader + round_up(rows * sizeof(float), 256) + round_up(rows * 3 * sizeof(float), 256) +
-               round_up((size_t)kRouterBwdChunks * (s->D > 0 ? s->D : 0) * 3 * sizeof(float), 256);
+               round_up((size_t)kRouterBwdChunks * (s->D > 0 ? s->D : 0) * 3 * sizeof(float), 256) +
+               round_up(bwd_stats_bytes(s), 256);
     }
     return 0;
 }
@@ -256,11 +263,17 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     p.Gpart = reinterpret_cast<float*>(w);
     w += round_up(rows * 3 * sizeof(float), 256);
     float* rpart = reinterpret_cast<float*>(w);
+    w += round_up((size_t)kRouterBwdChunks * (s->D > 0 ? s->D : 0) * 3 * sizeof(float), 256);
+    p.stats = reinterpret_cast<float*>(w);
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
     p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
-    cudaError_t e = launch_bwd_simt(p, s->dtype, cs);
+    cudaError_t e;
+    if (!(s->flags & MKA_FLAG_FORCE_SIMT) && bwd_tc_eligible(p, s->dtype))
+        e = launch_bwd_tc(p, static_cast<unsigned int*>(ws), cs);
+    else
+        e = launch_bwd_simt(p, s->dtype, cs);
     if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return MKA_ERR_CUDA;
     if (dW_r || db_r) {
@@ -268,6 +281,20 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
         if (e != cudaSuccess) return MKA_ERR_CUDA;
     }
     return MKA_OK;
+}
+
+int32_t mka_bwd_kernel_kind(const mka_shape* s, const mka_level L[3], const mka_level_grad dL[3]) {
+    if (check_shape(s, false) != MKA_OK || check_levels(s, L) != MKA_OK || s->mode != MKA_MODE_FAST) return -1;
+    BwdParams p;
+    memset(&p, 0, sizeof(p));
+    fill_levels(p.L, L);
+    for (int l = 0; l < 3; ++l) {
+        p.dL[l].sn = dL ? dL[l].stride_n : L[l].stride_n;
+        p.dL[l].sh = dL ? dL[l].stride_h : L[l].stride_h;
+        p.dL[l].sb = dL ? dL[l].stride_b : L[l].stride_b;
+    }
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
+    return (!(s->flags & MKA_FLAG_FORCE_SIMT) && bwd_tc_eligible(p, s->dtype)) ? 1 : 0;
 }
 
 mka_status mka_device_status(const void* ws, void* stream) {

@@ -285,6 +285,17 @@ __global__ void bwd_dgate_kernel(const float* __restrict__ Gpart, int B, int H, 
     dG[i] = s;
 }
 
+}  // namespace
+
+cudaError_t launch_bwd_dgate(const float* Gpart, int B, int H, long long T, float* dG, cudaStream_t st) {
+    const long long n = (long long)B * T * 3;
+    if (n == 0) return cudaSuccess;
+    bwd_dgate_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(Gpart, B, H, T, dG);
+    return cudaGetLastError();
+}
+
+namespace {
+
 template <typename T, int DH>
 cudaError_t launch_t(const BwdParams& p, cudaStream_t st) {
     const long long rows = (long long)p.B * p.H * p.T;
@@ -310,9 +321,7 @@ cudaError_t launch_t(const BwdParams& p, cudaStream_t st) {
             if ((e = cudaGetLastError()) != cudaSuccess) return e;
         }
     }
-    const long long n = (long long)p.B * p.T * 3;
-    bwd_dgate_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(p.Gpart, p.B, p.H, p.T, p.dG);
-    return cudaGetLastError();
+    return launch_bwd_dgate(p.Gpart, p.B, p.H, p.T, p.dG, st);
 }
 
 template <typename T>

@@ -1,0 +1,699 @@
+// Tensor-core backward of Eq. 5 for bf16 on sm_100a: TMA -> shared memory -> tcgen05.mma -> TMEM.
+//
+// The paper prints no backward; this one follows from differentiating Eq. 5.  With
+//   p = lambda_{t,l} exp(s - LSE_t) on the visible set,  dP = dO_t . v_{l,j},  D_t = dO_t . O_t,
+//   dS = p (dP - D_t):
+//     dV_{l,j} = sum_t p dO_t      dK_{l,j} = tau sum_t dS q_t      dQ_t = tau sum_{l,j} dS k_{l,j}
+//     G_{t,l}  = sum_{j in l} dS   (gradient of the router logit of level l, per head)
+//
+// Three launches, each deterministic (every output element has one owner, fixed summation order):
+//   bwd_prep_kernel    per (b,h,t): D_t and, per level, the exponent bias log2(lambda) - LSE log2(e)
+//   bwd_dq_tc_kernel   CTA = 128 query rows of one (b,h); streams the level-ordered list of 64-row
+//                      key sub-tiles (L1 window, L2 prefix, L3 slots) exactly like the forward:
+//                      S = Q K^T, dP = dO V^T (128x64 each), dS -> TMEM (bf16), dQ += dS K.
+//   bwd_dkv_tc_kernel  CTA = 128 key rows of one level of one (b,h); streams the 64-row query
+//                      sub-tiles that can see them: S^T = K Q^T, dP^T = V dO^T (128x64 each),
+//                      P^T, dS^T -> TMEM (bf16), dV += P^T dO, dK += dS^T Q.
+// Both kernels recompute the scores (7 matrix products per visible tile pair instead of 5) in exchange
+// for needing no atomics and no cross-CTA reduction.
+//
+// Warp roles (320 threads): warps 0-3 and 4-7 are two softmax warpgroups (thread i <-> TMEM lane i);
+// warpgroup w takes the sub-tiles with index = w (mod 2), which live in TMEM stage w, so the element-wise
+// work of one sub-tile overlaps the matrix products of the next.  Warp 8 lane 0 issues the TMA loads,
+// warp 9 lane 0 issues every tcgen05.mma.  TMEM: stage w holds S (64 columns) and dP (64 columns) of
+// a sub-tile; the bf16 results overwrite the first 32 columns of each; the fp32 accumulators follow.
+// Every mbarrier wait is bounded; on expiry the CTA raises a flag, drains and reports MKA_ERR_TIMEOUT.
+#include "tc_ptx.cuh"
+
+namespace mka {
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kSub = 64;                              // rows of a streamed sub-tile
+constexpr uint32_t kPanel128 = 128 * 128;             // bytes of a [128 rows][64 bf16] panel
+constexpr uint32_t kPanel64 = 64 * 128;               // bytes of a [64 rows][64 bf16] panel
+constexpr int kMaxStages = 8;
+
+struct BwdMaps {
+    CUtensorMap q, dO;
+    CUtensorMap k[3], v[3];
+};
+
+struct BwdTcParams {
+    __nv_bfloat16* dQ;
+    const float2* stats[3];   // per level: [B*H, Tpad] of {D_t, log2(lambda_{t,l}) - LSE_t log2(e)}
+    float* Gpart;             // [B, H, T, 3]
+    LevelGradDev dL[3];
+    long long n[3];
+    int B, H, T, Tpad;
+    int window, q_offset;
+    float scale, scale_log2;
+    int kv_tiles[3];          // 128-row key tiles per level
+    unsigned int* status;
+};
+
+template <int DH>
+struct BCfg {
+    static constexpr int kPanels = DH / 64;
+    static constexpr uint32_t kBig = kPanels * kPanel128;     // a 128-row tile
+    static constexpr uint32_t kSmall = kPanels * kPanel64;    // a 64-row sub-tile
+    static constexpr int kStages = DH == 128 ? 4 : 8;         // also keeps the CTA above half of shared memory
+    static constexpr uint32_t kStatBytes = kSub * sizeof(float2);
+    static constexpr uint32_t kSmemDq = 2 * kBig + kStages * 2 * kSmall + 1024;
+    static constexpr uint32_t kSmemDkv = 2 * kBig + kStages * (2 * kSmall + kStatBytes) + 1024;
+    // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
+    static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSub >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    static constexpr uint32_t kIdescAcc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    static constexpr uint32_t kAccCol = 256;                  // first accumulator column
+};
+
+struct BwdBarriers {
+    uint64_t fixed_full;                                  // the CTA's own (non-streamed) tiles
+    uint64_t a_full[kMaxStages], a_empty[kMaxStages];     // streamed operand ring (first stream)
+    uint64_t b_full[kMaxStages], b_empty[kMaxStages];     // streamed operand ring (second stream; dQ kernel only)
+    uint64_t sdp_full[2], ds_full[2];
+    uint64_t acc_done;
+};
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------ prep
+// One warp per padded row: D = dO . O and the three exponent biases.  Padding rows (t >= T) get a bias
+// of -inf so that a streamed sub-tile may run past the last query without a mask.
+template <int DH>
+__global__ void __launch_bounds__(256) bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
+                                                       const float* __restrict__ LSE, const float* __restrict__ gate, int H,
+                                                       int T, int Tpad, long long rows_pad, float2* __restrict__ s0,
+                                                       float2* __restrict__ s1, float2* __restrict__ s2) {
+    const int lane = threadIdx.x & 31;
+    const long long r = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (r >= rows_pad) return;
+    const long long bh = r / Tpad;
+    const int t = (int)(r % Tpad);
+    float2 o0 = make_float2(0.f, -INFINITY), o1 = o0, o2 = o0;
+    if (t < T) {
+        const long long row = bh * T + t;
+        constexpr int PER = DH / 32;                   // 2 or 4 consecutive elements per lane
+        const __nv_bfloat16* po = O + row * DH + lane * PER;
+        const __nv_bfloat16* pg = dO + row * DH + lane * PER;
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < PER; i += 2) {
+            const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(po + i);
+            const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(pg + i);
+            s = fmaf(__bfloat162float(a.x), __bfloat162float(g.x), s);
+            s = fmaf(__bfloat162float(a.y), __bfloat162float(g.y), s);
+        }
+        s = warp_sum(s);
+        const float lse = LSE[row];
+        const float* g = gate + ((bh / H) * T + t) * 3;
+        const bool live = lse > -INFINITY;
+        const float l2 = lse * kLog2e;
+        o0 = make_float2(s, (live && g[0] > 0.f) ? log2f(g[0]) - l2 : -INFINITY);
+        o1 = make_float2(s, (live && g[1] > 0.f) ? log2f(g[1]) - l2 : -INFINITY);
+        o2 = make_float2(s, (live && g[2] > 0.f) ? log2f(g[2]) - l2 : -INFINITY);
+    }
+    if (lane == 0) { s0[r] = o0; s1[r] = o1; s2[r] = o2; }
+}
+
+// Key sub-tile range [first, end) (64-row units) of query rows [r0, r1] on one level.
+__device__ __forceinline__ void sub_range(int level, long long r0, long long r1, int q_offset, int window, long long n,
+                                          int& first, int& end) {
+    long long lo_f, hi_f, lo_l, hi_l;
+    visible_range(level, r0 + q_offset, window, n, 0, lo_f, hi_f);
+    visible_range(level, r1 + q_offset, window, n, 0, lo_l, hi_l);
+    const long long hi = hi_l > hi_f ? hi_l : hi_f;
+    if (hi <= lo_f) { first = end = 0; return; }
+    first = (int)(lo_f / kSub);
+    end = (int)((hi + kSub - 1) / kSub);
+}
+
+__device__ __forceinline__ void store_row_bf16(__nv_bfloat16* dst, const uint32_t (&o)[32], float mul) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(o[i]) * mul, __uint_as_float(o[i + 1]) * mul);
+        v.y = pack_bf16(__uint_as_float(o[i + 2]) * mul, __uint_as_float(o[i + 3]) * mul);
+        v.z = pack_bf16(__uint_as_float(o[i + 4]) * mul, __uint_as_float(o[i + 5]) * mul);
+        v.w = pack_bf16(__uint_as_float(o[i + 6]) * mul, __uint_as_float(o[i + 7]) * mul);
+        *reinterpret_cast<uint4*>(dst + i) = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------ dQ
+template <int DH>
+__global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdTcParams p) {
+    using C = BCfg<DH>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* sQ = smem;
+    uint8_t* sdO = sQ + C::kBig;
+    uint8_t* sK = sdO + C::kBig;                          // kStages sub-tiles
+    uint8_t* sV = sK + C::kStages * C::kSmall;            // kStages sub-tiles
+    __shared__ BwdBarriers bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ float gsm[128][6];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.z, h = blockIdx.y;
+    const long long bh = (long long)b * p.H + h;
+    const int qtile = gridDim.x - 1 - blockIdx.x;          // latest (heaviest) rows first
+    const long long m0 = (long long)qtile * 128;
+    const long long m_last = (m0 + 127 < p.T - 1) ? m0 + 127 : p.T - 1;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(&bar.fixed_full, 1);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1);
+            mbar_init(&bar.b_full[s], 1); mbar_init(&bar.b_empty[s], 1);
+        }
+        for (int w = 0; w < 2; ++w) { mbar_init(&bar.sdp_full[w], 1); mbar_init(&bar.ds_full[w], 128); }
+        mbar_init(&bar.acc_done, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    int first[3], end[3];
+#pragma unroll
+    for (int l = 0; l < 3; ++l) {
+        if (p.n[l] > 0) sub_range(l, m0, m_last, p.q_offset, p.window, p.n[l], first[l], end[l]);
+        else first[l] = end[l] = 0;
+    }
+    const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
+
+    if (warp == kProducerWarp) {
+        if (lane == 0) {
+            mbar_expect_tx(&bar.fixed_full, 2 * C::kBig);
+#pragma unroll
+            for (int pn = 0; pn < C::kPanels; ++pn) {
+                tma_load_4d(sQ + pn * kPanel128, &maps.q, pn * 64, (int)m0, h, b, &bar.fixed_full);
+                tma_load_4d(sdO + pn * kPanel128, &maps.dO, pn * 64, (int)m0, h, b, &bar.fixed_full);
+            }
+            int issued_k = 0, issued_v = 0;
+            bool ok = true;
+            for (int l = 0; l < 3 && ok; ++l) {
+                for (int kt = first[l]; kt < end[l]; ++kt) {
+                    const int s = issued_k % C::kStages;
+                    const uint32_t ph = (uint32_t)(issued_k / C::kStages) & 1u;
+                    if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
+                    mbar_expect_tx(&bar.a_full[s], C::kSmall);
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sK + s * C::kSmall + pn * kPanel64, &maps.k[l], pn * 64, kt * kSub, h, b, &bar.a_full[s]);
+                    ++issued_k;
+                    if (!mbar_wait(&bar.b_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
+                    mbar_expect_tx(&bar.b_full[s], C::kSmall);
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sV + s * C::kSmall + pn * kPanel64, &maps.v[l], pn * 64, kt * kSub, h, b, &bar.b_full[s]);
+                    ++issued_v;
+                }
+            }
+            // every copy issued above must have landed before the shared memory can be given up
+            mbar_wait(&bar.fixed_full, 0, abortp);
+            for (int i = issued_k > C::kStages ? issued_k - C::kStages : 0; i < issued_k; ++i)
+                mbar_wait(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+            for (int i = issued_v > C::kStages ? issued_v - C::kStages : 0; i < issued_v; ++i)
+                mbar_wait(&bar.b_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane == 0) {
+            bool ok = mbar_wait(&bar.fixed_full, 0, abortp);
+            tc_fence_after();
+            const uint32_t q_addr = smem_u32(sQ), g_addr = smem_u32(sdO), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+            auto issue_dq = [&](int e) -> bool {           // dQ += dS(e) K(e)
+                const int w = e & 1, s = e % C::kStages;
+                if (!mbar_wait(&bar.ds_full[w], (uint32_t)(e >> 1) & 1u, abortp)) return false;
+                tc_fence_after();
+                const uint32_t ka = k_addr + s * C::kSmall;
+#pragma unroll
+                for (int k = 0; k < kSub / 16; ++k)
+                    mma_ts(tmem + C::kAccCol, tmem + w * 128 + k * 8, desc_mnmajor(ka + k * 2048, kPanel64), C::kIdescAcc,
+                           (e > 0 || k > 0) ? 1u : 0u);
+                mma_commit(&bar.a_empty[s]);
+                return true;
+            };
+            for (int e = 0; e < E && ok; ++e) {
+                const int w = e & 1, s = e % C::kStages;
+                const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                if (!mbar_wait(&bar.a_full[s], ph, abortp) || !mbar_wait(&bar.b_full[s], ph, abortp)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t ka = k_addr + s * C::kSmall, va = v_addr + s * C::kSmall;
+#pragma unroll
+                for (int k = 0; k < DH / 16; ++k)          // S = Q K^T
+                    mma_ss(tmem + w * 128, desc_kmajor(q_addr + (k / 4) * kPanel128 + (k % 4) * 32),
+                           desc_kmajor(ka + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
+#pragma unroll
+                for (int k = 0; k < DH / 16; ++k)          // dP = dO V^T
+                    mma_ss(tmem + w * 128 + 64, desc_kmajor(g_addr + (k / 4) * kPanel128 + (k % 4) * 32),
+                           desc_kmajor(va + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
+                mma_commit(&bar.sdp_full[w]);
+                mma_commit(&bar.b_empty[s]);
+                if (e > 0 && !issue_dq(e - 1)) { ok = false; break; }
+            }
+            if (ok && E > 0 && issue_dq(E - 1)) mma_commit(&bar.acc_done);
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warpgroups
+        const int w = warp >> 2;
+        const int r = tid & 127;
+        const long long t = m0 + r;
+        const bool row_valid = t < p.T;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t st_addr = tmem + lane_base + w * 128;
+        float Dt = 0.f, bias[3] = {-INFINITY, -INFINITY, -INFINITY};
+        if (row_valid) {
+#pragma unroll
+            for (int l = 0; l < 3; ++l) {
+                const float2 sv = p.stats[l][bh * p.Tpad + t];
+                Dt = sv.x;
+                bias[l] = sv.y;
+            }
+        }
+        float Al[3] = {0.f, 0.f, 0.f}, Sl[3] = {0.f, 0.f, 0.f};   // per level: sum p dP and sum p
+        bool ok = true;
+        int e = 0;
+#pragma unroll
+        for (int l = 0; l < 3; ++l) {
+            if (!ok || first[l] == end[l]) continue;
+            long long lo = 0, hi = 0;
+            if (row_valid) visible_range(l, t + p.q_offset, p.window, p.n[l], 0, lo, hi);
+            int full_first = 0, full_end = 0;
+            {
+                long long lo_f, hi_f, lo_l, hi_l;
+                visible_range(l, m0 + p.q_offset, p.window, p.n[l], 0, lo_f, hi_f);
+                visible_range(l, m_last + p.q_offset, p.window, p.n[l], 0, lo_l, hi_l);
+                full_first = (int)((lo_l + kSub - 1) / kSub);
+                full_end = (int)(hi_f / kSub);
+                if (m_last - m0 + 1 < 128) full_end = full_first;           // ragged query tile: always mask
+            }
+            float a0 = 0.f, a1 = 0.f, z0 = 0.f, z1 = 0.f;
+            for (int kt = first[l]; kt < end[l]; ++kt, ++e) {
+                if ((e & 1) != w) continue;
+                ok = mbar_wait(&bar.sdp_full[w], (uint32_t)(e >> 1) & 1u, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                float s[kSub], dp[kSub];
+                tmem_ld32(st_addr, reinterpret_cast<uint32_t*>(s));
+                tmem_ld32(st_addr + 32, reinterpret_cast<uint32_t*>(s) + 32);
+                tmem_ld32(st_addr + 64, reinterpret_cast<uint32_t*>(dp));
+                tmem_ld32(st_addr + 96, reinterpret_cast<uint32_t*>(dp) + 32);
+                tmem_ld_wait();
+                if (!(kt >= full_first && kt < full_end)) {
+                    const int c_lo = (int)max(-1LL, min(lo - (long long)kt * kSub, (long long)kSub));
+                    const int c_hi = (int)max(-1LL, min(hi - (long long)kt * kSub, (long long)kSub));
+#pragma unroll
+                    for (int c = 0; c < kSub; ++c)
+                        if (c < c_lo || c >= c_hi) s[c] = -INFINITY;
+                }
+                uint32_t pk[kSub / 2];
+                const float bl = bias[l];
+#pragma unroll
+                for (int c = 0; c < kSub; c += 2) {
+                    const float p0 = ex2(fmaf(s[c], p.scale_log2, bl));
+                    const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, bl));
+                    a0 = fmaf(p0, dp[c], a0);
+                    a1 = fmaf(p1, dp[c + 1], a1);
+                    z0 += p0;
+                    z1 += p1;
+                    pk[c / 2] = pack_bf16(p0 * (dp[c] - Dt), p1 * (dp[c + 1] - Dt));
+                }
+                tmem_st32(st_addr, pk);
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&bar.ds_full[w]);
+            }
+            Al[l] = a0 + a1;
+            Sl[l] = z0 + z1;
+        }
+        // ------------------------------------------------------------ epilogue
+        if (ok && E > 0) {
+            ok = mbar_wait(&bar.acc_done, 0, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            __nv_bfloat16* out = p.dQ + (bh * p.T + t) * DH;
+#pragma unroll
+            for (int c0 = w * (DH / 2); c0 < (w + 1) * (DH / 2); c0 += 32) {
+                uint32_t o[32];
+                if (E > 0) {
+                    tmem_ld32(tmem + lane_base + C::kAccCol + c0, o);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = 0u;
+                }
+                if (row_valid) store_row_bf16(out + c0, o, p.scale);
+            }
+        }
+        // Gate-logit gradient of this head: G_l = sum_{j in l} p (dP - D').  D' = sum p dP / sum p equals
+        // dO . O in exact arithmetic but does not inherit the rounding of O to bf16, so sum_l G_l = 0 holds
+        // to fp32 accuracy.  The two warpgroups hold disjoint sub-tiles: add their partial sums first.
+        if (w == 1) {
+#pragma unroll
+            for (int l = 0; l < 3; ++l) { gsm[r][l] = Al[l]; gsm[r][3 + l] = Sl[l]; }
+        }
+        softmax_group_sync();
+        if (w == 0 && ok && row_valid) {
+            float a[3], z[3];
+#pragma unroll
+            for (int l = 0; l < 3; ++l) { a[l] = Al[l] + gsm[r][l]; z[l] = Sl[l] + gsm[r][3 + l]; }
+            const float ztot = z[0] + z[1] + z[2];
+            const float dd = ztot > 0.f ? (a[0] + a[1] + a[2]) / ztot : 0.f;
+            float* g = p.Gpart + (bh * p.T + t) * 3;
+#pragma unroll
+            for (int l = 0; l < 3; ++l) g[l] = a[l] - z[l] * dd;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------ dK, dV
+template <int DH>
+__global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdTcParams p) {
+    using C = BCfg<DH>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* sK = smem;
+    uint8_t* sV = sK + C::kBig;
+    uint8_t* sQ = sV + C::kBig;                           // kStages sub-tiles
+    uint8_t* sdO = sQ + C::kStages * C::kSmall;           // kStages sub-tiles
+    float2* sStat = reinterpret_cast<float2*>(sdO + C::kStages * C::kSmall);   // kStages x 64
+    __shared__ BwdBarriers bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.z, h = blockIdx.y;
+    const long long bh = (long long)b * p.H + h;
+    // key tiles in decreasing order of work: L3 (seen by every query), L2 from the oldest key on, L1
+    int lvl, kt;
+    {
+        int x = blockIdx.x;
+        if (x < p.kv_tiles[2]) { lvl = 2; kt = x; }
+        else if (x < p.kv_tiles[2] + p.kv_tiles[1]) { lvl = 1; kt = x - p.kv_tiles[2]; }
+        else { lvl = 0; kt = x - p.kv_tiles[2] - p.kv_tiles[1]; }
+    }
+    const long long n = p.n[lvl];
+    const long long j0 = (long long)kt * 128;
+    const long long j_last = (j0 + 127 < n - 1) ? j0 + 127 : n - 1;
+    // queries t (position t + q_offset) that can see a key of this tile
+    long long t_lo = 0, t_hi = p.T;
+    if (lvl == 0) { t_lo = j0 - p.q_offset; t_hi = j_last + p.window - p.q_offset; }
+    else if (lvl == 1) { t_lo = j0 - p.q_offset; }
+    if (t_lo < 0) t_lo = 0;
+    if (t_hi > p.T) t_hi = p.T;
+    const int first = t_hi > t_lo ? (int)(t_lo / kSub) : 0;
+    const int E = t_hi > t_lo ? (int)((t_hi + kSub - 1) / kSub) - first : 0;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(&bar.fixed_full, 1);
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1); }
+        for (int w = 0; w < 2; ++w) { mbar_init(&bar.sdp_full[w], 1); mbar_init(&bar.ds_full[w], 128); }
+        mbar_init(&bar.acc_done, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    if (warp == kProducerWarp) {
+        if (lane == 0) {
+            bool ok = true;
+            int issued = 0;
+            if (E > 0) {
+                mbar_expect_tx(&bar.fixed_full, 2 * C::kBig);
+#pragma unroll
+                for (int pn = 0; pn < C::kPanels; ++pn) {
+                    tma_load_4d(sK + pn * kPanel128, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                    tma_load_4d(sV + pn * kPanel128, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                }
+                const float2* stat = p.stats[lvl] + bh * p.Tpad;
+                for (int e = 0; e < E; ++e) {
+                    const int s = e % C::kStages;
+                    const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                    if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
+                    const int tt = (first + e) * kSub;
+                    mbar_expect_tx(&bar.a_full[s], 2 * C::kSmall + C::kStatBytes);
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn) {
+                        tma_load_4d(sQ + s * C::kSmall + pn * kPanel64, &maps.q, pn * 64, tt, h, b, &bar.a_full[s]);
+                        tma_load_4d(sdO + s * C::kSmall + pn * kPanel64, &maps.dO, pn * 64, tt, h, b, &bar.a_full[s]);
+                    }
+                    bulk_load(sStat + s * kSub, stat + tt, C::kStatBytes, &bar.a_full[s]);
+                    ++issued;
+                }
+                mbar_wait(&bar.fixed_full, 0, abortp);
+                for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
+                    mbar_wait(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+            }
+            (void)ok;
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane == 0 && E > 0) {
+            bool ok = mbar_wait(&bar.fixed_full, 0, abortp);
+            tc_fence_after();
+            const uint32_t k_addr = smem_u32(sK), v_addr = smem_u32(sV), q_addr = smem_u32(sQ), g_addr = smem_u32(sdO);
+            auto issue_acc = [&](int e) -> bool {          // dV += P^T(e) dO(e);  dK += dS^T(e) Q(e)
+                const int w = e & 1, s = e % C::kStages;
+                if (!mbar_wait(&bar.ds_full[w], (uint32_t)(e >> 1) & 1u, abortp)) return false;
+                tc_fence_after();
+                const uint32_t qa = q_addr + s * C::kSmall, ga = g_addr + s * C::kSmall;
+#pragma unroll
+                for (int k = 0; k < kSub / 16; ++k)
+                    mma_ts(tmem + C::kAccCol + DH, tmem + w * 128 + k * 8, desc_mnmajor(ga + k * 2048, kPanel64), C::kIdescAcc,
+                           (e > 0 || k > 0) ? 1u : 0u);
+#pragma unroll
+                for (int k = 0; k < kSub / 16; ++k)
+                    mma_ts(tmem + C::kAccCol, tmem + w * 128 + 64 + k * 8, desc_mnmajor(qa + k * 2048, kPanel64), C::kIdescAcc,
+                           (e > 0 || k > 0) ? 1u : 0u);
+                mma_commit(&bar.a_empty[s]);
+                return true;
+            };
+            for (int e = 0; e < E && ok; ++e) {
+                const int w = e & 1, s = e % C::kStages;
+                const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                if (!mbar_wait(&bar.a_full[s], ph, abortp)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t qa = q_addr + s * C::kSmall, ga = g_addr + s * C::kSmall;
+#pragma unroll
+                for (int k = 0; k < DH / 16; ++k)          // S^T = K Q^T
+                    mma_ss(tmem + w * 128, desc_kmajor(k_addr + (k / 4) * kPanel128 + (k % 4) * 32),
+                           desc_kmajor(qa + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
+#pragma unroll
+                for (int k = 0; k < DH / 16; ++k)          // dP^T = V dO^T
+                    mma_ss(tmem + w * 128 + 64, desc_kmajor(v_addr + (k / 4) * kPanel128 + (k % 4) * 32),
+                           desc_kmajor(ga + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
+                mma_commit(&bar.sdp_full[w]);
+                if (e > 0 && !issue_acc(e - 1)) { ok = false; break; }
+            }
+            if (ok && issue_acc(E - 1)) mma_commit(&bar.acc_done);
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warpgroups (thread = key row)
+        const int w = warp >> 2;
+        const int r = tid & 127;
+        const long long j = j0 + r;
+        const bool row_valid = j < n;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t st_addr = tmem + lane_base + w * 128;
+        // queries [q_lo, q_hi) that see key j (the bound t < T is carried by the padded biases)
+        long long q_lo = 0, q_hi = 0;
+        if (row_valid) {
+            q_lo = lvl == 2 ? 0 : j - p.q_offset;
+            q_hi = lvl == 0 ? j + p.window - p.q_offset : (long long)p.Tpad;
+        }
+        // sub-tiles whose every (key, query) pair is visible need no mask
+        const bool rows_full = j0 + 127 < n;
+        bool ok = true;
+        for (int e = w; e < E; e += 2) {
+            const int s = e % C::kStages;
+            const long long tt = (long long)(first + e) * kSub;
+            ok = mbar_wait(&bar.sdp_full[w], (uint32_t)(e >> 1) & 1u, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float sc[kSub], dp[kSub];
+            tmem_ld32(st_addr, reinterpret_cast<uint32_t*>(sc));
+            tmem_ld32(st_addr + 32, reinterpret_cast<uint32_t*>(sc) + 32);
+            tmem_ld32(st_addr + 64, reinterpret_cast<uint32_t*>(dp));
+            tmem_ld32(st_addr + 96, reinterpret_cast<uint32_t*>(dp) + 32);
+            tmem_ld_wait();
+            bool full = rows_full;
+            if (lvl != 2) full = full && (j_last - p.q_offset <= tt);
+            if (lvl == 0) full = full && (j0 + p.window - p.q_offset >= tt + kSub);
+            if (!full) {
+                const int c_lo = (int)max(-1LL, min(q_lo - tt, (long long)kSub));
+                const int c_hi = (int)max(-1LL, min(q_hi - tt, (long long)kSub));
+#pragma unroll
+                for (int c = 0; c < kSub; ++c)
+                    if (c < c_lo || c >= c_hi) sc[c] = -INFINITY;
+            }
+            const float4* stat = reinterpret_cast<const float4*>(sStat + s * kSub);   // two queries per load
+            uint32_t pkP[kSub / 2], pkD[kSub / 2];
+#pragma unroll
+            for (int c = 0; c < kSub; c += 2) {
+                const float4 sv = stat[c / 2];                                          // {D_c, bias_c, D_c+1, bias_c+1}
+                const float p0 = ex2(fmaf(sc[c], p.scale_log2, sv.y));
+                const float p1 = ex2(fmaf(sc[c + 1], p.scale_log2, sv.w));
+                pkP[c / 2] = pack_bf16(p0, p1);
+                pkD[c / 2] = pack_bf16(p0 * (dp[c] - sv.x), p1 * (dp[c + 1] - sv.z));
+            }
+            tmem_st32(st_addr, pkP);
+            tmem_st32(st_addr + 64, pkD);
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(&bar.ds_full[w]);
+        }
+        // ------------------------------------------------------------ epilogue: warpgroup 0 writes dK, 1 writes dV
+        if (ok && E > 0) {
+            ok = mbar_wait(&bar.acc_done, 0, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const LevelGradDev dL = p.dL[lvl];
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(w == 0 ? dL.dk : dL.dv) + b * dL.sb + h * dL.sh + j * dL.sn;
+            const float mul = w == 0 ? p.scale : 1.f;
+#pragma unroll
+            for (int c0 = 0; c0 < DH; c0 += 32) {
+                uint32_t o[32];
+                if (E > 0) {
+                    tmem_ld32(tmem + lane_base + C::kAccCol + w * DH + c0, o);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = 0u;
+                }
+                if (row_valid) store_row_bf16(out + c0, o, mul);
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+}
+
+template <int DH>
+cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_t st) {
+    using C = BCfg<DH>;
+    const int Tpad = (bp.T + kSub - 1) / kSub * kSub;
+    const long long rows_pad = (long long)bp.B * bp.H * Tpad;
+    float2* stats[3];
+    for (int l = 0; l < 3; ++l) stats[l] = reinterpret_cast<float2*>(bp.stats) + (long long)l * rows_pad;
+    const long long sq_n = DH, sq_h = (long long)bp.T * DH, sq_b = (long long)bp.H * bp.T * DH;
+
+    bwd_prep_kernel<DH><<<(unsigned)((rows_pad + 7) / 8), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(bp.O), static_cast<const __nv_bfloat16*>(bp.dO), bp.LSE, bp.gate, bp.H, bp.T, Tpad,
+        rows_pad, stats[0], stats[1], stats[2]);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+
+    BwdTcParams p;
+    p.dQ = static_cast<__nv_bfloat16*>(bp.dQ);
+    p.Gpart = bp.Gpart;
+    for (int l = 0; l < 3; ++l) {
+        p.stats[l] = stats[l];
+        p.dL[l] = bp.dL[l];
+        p.n[l] = bp.L[l].n;
+        p.kv_tiles[l] = (int)((bp.L[l].n + 127) / 128);
+    }
+    p.B = bp.B; p.H = bp.H; p.T = bp.T; p.Tpad = Tpad;
+    p.window = bp.window; p.q_offset = bp.q_offset;
+    p.scale = bp.scale; p.scale_log2 = bp.scale * kLog2e;
+    p.status = status_word;
+
+    // dQ: 128-row Q / dO tiles, 64-row key sub-tiles
+    {
+        BwdMaps m;
+        if (!make_bf16_map(&m.q, bp.Q, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, 128) ||
+            !make_bf16_map(&m.dO, bp.dO, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, 128))
+            return cudaErrorNotSupported;
+        for (int l = 0; l < 3; ++l) {
+            if (bp.L[l].n == 0) { m.k[l] = m.q; m.v[l] = m.q; continue; }
+            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kSub) ||
+                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kSub))
+                return cudaErrorNotSupported;
+        }
+        e = cudaFuncSetAttribute(bwd_dq_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemDq);
+        if (e != cudaSuccess) return e;
+        dim3 grid((bp.T + 127) / 128, bp.H, bp.B);
+        bwd_dq_tc_kernel<DH><<<grid, kThreads, C::kSmemDq, st>>>(m, p);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    // dK, dV: 128-row key tiles, 64-row Q / dO sub-tiles
+    const int tiles = p.kv_tiles[0] + p.kv_tiles[1] + p.kv_tiles[2];
+    if (tiles > 0) {
+        BwdMaps m;
+        if (!make_bf16_map(&m.q, bp.Q, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, kSub) ||
+            !make_bf16_map(&m.dO, bp.dO, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, kSub))
+            return cudaErrorNotSupported;
+        for (int l = 0; l < 3; ++l) {
+            if (bp.L[l].n == 0) { m.k[l] = m.q; m.v[l] = m.q; continue; }
+            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, 128) ||
+                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, 128))
+                return cudaErrorNotSupported;
+        }
+        e = cudaFuncSetAttribute(bwd_dkv_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemDkv);
+        if (e != cudaSuccess) return e;
+        dim3 grid(tiles, bp.H, bp.B);
+        bwd_dkv_tc_kernel<DH><<<grid, kThreads, C::kSmemDkv, st>>>(m, p);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    return launch_bwd_dgate(bp.Gpart, bp.B, bp.H, bp.T, bp.dG, st);
+}
+
+}  // namespace
+
+bool bwd_tc_eligible(const BwdParams& p, int dtype) {
+    if (dtype != MKA_BF16) return false;
+    if (p.d != 64 && p.d != 128) return false;
+    if (p.H > 65535 || p.B > 65535) return false;
+    for (int l = 0; l < 3; ++l) {
+        const LevelDev& L = p.L[l];
+        if (L.n == 0) continue;
+        if (L.n > 0x7fffffffLL - 256) return false;
+        if (L.sn % 8 || L.sn <= 0) return false;
+        if (p.H > 1 && (L.sh % 8 || L.sh <= 0)) return false;
+        if (p.B > 1 && (L.sb % 8 || L.sb <= 0)) return false;
+        if (p.dL[l].sn % 8 || p.dL[l].sh % 8 || p.dL[l].sb % 8) return false;
+    }
+    return tensor_map_encoder_available();
+}
+
+cudaError_t launch_bwd_tc(const BwdParams& p, unsigned int* status_word, cudaStream_t st) {
+    if (p.B == 0 || p.H == 0 || p.T == 0) return cudaSuccess;
+    return p.d == 128 ? launch_t<128>(p, status_word, st) : launch_t<64>(p, status_word, st);
+}
+
+}  // namespace mka

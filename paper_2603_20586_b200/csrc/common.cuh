@@ -110,6 +110,7 @@ struct BwdParams {
     float* dG;        // [B,T,3]
     float* delta;     // ws: [B,H,T]
     float* Gpart;     // ws: [B,H,T,3]
+    float* stats;     // ws: 3 x [B,H,Tpad] float2 (tensor-core path; Tpad = T rounded up to 64)
     int B, H, T, d;
     int window, q_offset;
     float scale;
@@ -117,6 +118,11 @@ struct BwdParams {
 cudaError_t launch_bwd_simt(const BwdParams& p, int dtype, cudaStream_t st);
 cudaError_t launch_router_bwd(const void* R, int r_dtype, const float* dG, long long rows, int D, float* dW_r,
                               float* db_r, float* partial, int n_row_chunks, cudaStream_t st);
+
+cudaError_t launch_bwd_dgate(const float* Gpart, int B, int H, long long T, float* dG, cudaStream_t st);
+// Tensor-core (TMA + tcgen05) backward; same contract as the forward below.
+cudaError_t launch_bwd_tc(const BwdParams& p, unsigned int* status_word, cudaStream_t st);
+bool bwd_tc_eligible(const BwdParams& p, int dtype);
 
 // Tensor-core (TMA + tcgen05) forward; returns cudaErrorNotSupported when the shape is not eligible.
 cudaError_t launch_fwd_tc(const FwdParams& p, unsigned int* status_word, cudaStream_t st);

@@ -205,21 +205,28 @@ BWD_CASES = [
     (1, 2, 200, 64, 64, 0, (200, 200, 130)),
     (2, 2, 96, 128, 200, 0, (96, 96, 0)),
     (1, 1, 70, 64, 30, 50, (120, 120, 33)),
+    (1, 2, 300, 128, 96, 0, (300, 300, 160)),       # several query tiles and key tiles, ragged tails
+    (1, 1, 333, 64, 100, 17, (400, 400, 65)),       # q_offset, window edge inside a sub-tile
+    (2, 1, 130, 128, 1, 0, (130, 130, 8)),          # window of one row, a few L3 slots
+    (1, 1, 257, 128, 64, 300, (600, 520, 0)),       # queries far from key 0: L1 starts past the first tiles
 ]
 
 
 @pytest.mark.parametrize("case", BWD_CASES)
-@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_bwd_matches_oracle(mka, orc, case, dtype):
+@pytest.mark.parametrize("dtype,flags", [(torch.bfloat16, 0), (torch.bfloat16, 1), (torch.float32, 0)])
+def test_bwd_matches_oracle(mka, orc, case, dtype, flags):
     B, H, T, d, W, q_off, N = case
     D = 48
     P = problem(37, B, H, T, d, N, D, dtype, router_std=0.3, with_dO=True)
     gate = mka.mka_router(P["X"], P["W_r"], None)
-    shape = mka.make_shape(B, H, T, d, D, W, q_off, dtype=_dt(mka, dtype))
+    shape = mka.make_shape(B, H, T, d, D, W, q_off, dtype=_dt(mka, dtype), flags=flags)
     O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
     K = [k if k.shape[2] else None for k in P["K"]]
     V = [v if v.shape[2] else None for v in P["V"]]
-    g = mka.mka_bwd(shape, P["Q"], K, V, gate, O, LSE, P["dO"], R=P["X"])
+    assert mka.mka_bwd_kernel_kind(shape, K, V) == (1 if dtype == torch.bfloat16 and flags == 0 else 0)
+    ws = mka.alloc_workspace(shape, N, mka.MKA_WS_BWD, "cuda")
+    g = mka.mka_bwd(shape, P["Q"], K, V, gate, O, LSE, P["dO"], R=P["X"], ws=ws)
+    assert mka.mka_device_status(ws) == 0
     torch.cuda.synchronize()
     rg, _ = orc.router(np64(P["X"]), np64(P["W_r"]))
     ref = orc.bwd(P["Q"], P["K"], P["V"], rg, P["dO"], W, q_off)
@@ -236,6 +243,56 @@ def test_bwd_matches_oracle(mka, orc, case, dtype):
     scale = max(1.0, float(np.abs(dW).max()))
     assert err(g["dW_r"], dW)[0] <= (5e-2 if dtype == torch.bfloat16 else 2e-4) * scale
     assert err(g["db_r"], db)[0] <= (5e-2 if dtype == torch.bfloat16 else 2e-4) * max(1.0, float(np.abs(db).max()))
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_bwd_one_hot_and_zero_gates(mka, orc, flags):
+    """A level whose gate is 0 gets exactly zero dK, dV; a one-hot gate is standard attention backward on that level."""
+    B, H, T, d, W, N = 1, 2, 200, 128, 50, (200, 200, 90)
+    P = problem(43, B, H, T, d, N, 32, torch.bfloat16, with_dO=True)
+    gate = torch.zeros(B, T, 3, device="cuda")
+    gate[:, : T // 2, 1] = 1.0                       # first half: L2 only
+    gate[:, T // 2:, 0] = 0.25                       # second half: L1 and L3, L2 off
+    gate[:, T // 2:, 2] = 0.75
+    shape = mka.make_shape(B, H, T, d, 32, W, flags=flags)
+    O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+    g = mka.mka_bwd(shape, P["Q"], P["K"], P["V"], gate, O, LSE, P["dO"])
+    ref = orc.bwd(P["Q"], P["K"], P["V"], np64(gate), P["dO"], W)
+    check(g["dQ"], ref["dQ"], torch.bfloat16, "dQ")
+    for l in range(3):
+        check(g["dK"][l], ref["dK"][l], torch.bfloat16, f"dK{l}")
+        check(g["dV"][l], ref["dV"][l], torch.bfloat16, f"dV{l}")
+    assert float(g["dK"][1][:, :, T // 2:].abs().max()) == 0.0     # L2 keys past row T/2 are seen only with gate 0
+    assert float(g["dV"][1][:, :, T // 2:].abs().max()) == 0.0
+    assert float(g["dG"][:, : T // 2].abs().max()) <= 1e-5           # one-hot rows: no gate gradient
+    assert err(g["dG"], ref["dG"])[0] <= 2e-2
+
+
+def test_bwd_strided_levels_and_gradients(mka, orc):
+    """K/V and their gradients as slices of larger buffers (explicit strides), tensor-core path."""
+    B, H, T, d, W, N = 2, 2, 150, 64, 40, (150, 150, 70)
+    P = problem(47, B, H, T, d, N, 32, torch.bfloat16, with_dO=True)
+    big = [torch.zeros(B, H, n + 24, d + 64, dtype=torch.bfloat16, device="cuda") for n in N]
+    bigv = [torch.zeros_like(x) for x in big]
+    K = [big[l][:, :, 8:8 + N[l], 16:16 + d] for l in range(3)]
+    V = [bigv[l][:, :, 8:8 + N[l], 16:16 + d] for l in range(3)]
+    for l in range(3):
+        K[l].copy_(P["K"][l]); V[l].copy_(P["V"][l])
+    gbig = [torch.full_like(x, 7.0) for x in big]
+    gbigv = [torch.full_like(x, 7.0) for x in big]
+    dK = [gbig[l][:, :, 8:8 + N[l], 16:16 + d] for l in range(3)]
+    dV = [gbigv[l][:, :, 8:8 + N[l], 16:16 + d] for l in range(3)]
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    shape = mka.make_shape(B, H, T, d, 32, W)
+    assert mka.mka_bwd_kernel_kind(shape, K, V) == 1
+    O, LSE = mka.mka_fwd(shape, P["Q"], K, V, gate)
+    g = mka.mka_bwd(shape, P["Q"], K, V, gate, O, LSE, P["dO"], dK=dK, dV=dV)
+    ref = orc.bwd(P["Q"], P["K"], P["V"], np64(gate), P["dO"], W)
+    for l in range(3):
+        check(dK[l], ref["dK"][l], torch.bfloat16, f"dK{l}")
+        check(dV[l], ref["dV"][l], torch.bfloat16, f"dV{l}")
+        assert float(gbig[l][:, :, :8].min()) == 7.0 and float(gbig[l][..., :16].min()) == 7.0   # nothing outside the slice
+    check(g["dQ"], ref["dQ"], torch.bfloat16, "dQ")
 
 
 def test_bwd_is_deterministic(mka):
