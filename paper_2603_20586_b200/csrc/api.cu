@@ -50,9 +50,9 @@ void fill_levels(LevelDev out[3], const mka_level L[3]) {
 
 constexpr int kRouterBwdChunks = 128;
 
-// Per-row statistics of the tensor-core backward: three arrays of [B, H, Tpad] float2, Tpad = T rounded up to 64.
+// Per-row statistics of the tensor-core backward: three arrays of [B, H, Tpad] float2, Tpad = T rounded up to 128.
 size_t bwd_stats_bytes(const mka_shape* s) {
-    const size_t tpad = ((size_t)s->T + 63) / 64 * 64;
+    const size_t tpad = ((size_t)s->T + 127) / 128 * 128;
     return (size_t)3 * s->B * s->H * tpad * 2 * sizeof(float);
 }
 

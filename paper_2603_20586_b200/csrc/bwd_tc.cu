@@ -8,20 +8,24 @@
 //
 // Three launches, each deterministic (every output element has one owner, fixed summation order):
 //   bwd_prep_kernel    per (b,h,t): D_t and, per level, the exponent bias log2(lambda) - LSE log2(e)
-//   bwd_dq_tc_kernel   CTA = 128 query rows of one (b,h); streams the level-ordered list of 64-row
-//                      key sub-tiles (L1 window, L2 prefix, L3 slots) exactly like the forward:
-//                      S = Q K^T, dP = dO V^T (128x64 each), dS -> TMEM (bf16), dQ += dS K.
-//   bwd_dkv_tc_kernel  CTA = 128 key rows of one level of one (b,h); streams the 64-row query
-//                      sub-tiles that can see them: S^T = K Q^T, dP^T = V dO^T (128x64 each),
-//                      P^T, dS^T -> TMEM (bf16), dV += P^T dO, dK += dS^T Q.
+//   bwd_dq_tc_kernel   CTA = 128 query rows of one (b,h); streams the level-ordered list of 128-row
+//                      key tiles (L1 window, L2 prefix, L3 slots) exactly like the forward:
+//                      S = Q K^T, dP = dO V^T (128x128 each), dS -> TMEM (bf16), dQ += dS K.
+//   bwd_dkv_tc_kernel  CTA = 128 key rows of one level of one (b,h); streams the 128-row query
+//                      tiles that can see them: S^T = K Q^T, dP^T = V dO^T, P^T and dS^T -> TMEM
+//                      (bf16), dV += P^T dO, dK += dS^T Q.
 // Both kernels recompute the scores (7 matrix products per visible tile pair instead of 5) in exchange
 // for needing no atomics and no cross-CTA reduction.
 //
-// Warp roles (320 threads): warps 0-3 and 4-7 are two softmax warpgroups (thread i <-> TMEM lane i);
-// warpgroup w takes the sub-tiles with index = w (mod 2), which live in TMEM stage w, so the element-wise
-// work of one sub-tile overlaps the matrix products of the next.  Warp 8 lane 0 issues the TMA loads,
-// warp 9 lane 0 issues every tcgen05.mma.  TMEM: stage w holds S (64 columns) and dP (64 columns) of
-// a sub-tile; the bf16 results overwrite the first 32 columns of each; the fp32 accumulators follow.
+// Warp roles (320 threads): warps 0-7 are the element-wise ("softmax") threads: thread i of either
+// warpgroup owns TMEM lane i & 127 (a query row in the dQ kernel, a key row in the dK/dV kernel);
+// warpgroup 0 takes columns 0-63 of a tile and warpgroup 1 columns 64-127.  Their work on a tile has
+// two phases so that it overlaps the tensor pipe: phase 1 needs only S (p = 2^(s*scale + bias), kept in
+// registers) and runs while dP is still being multiplied; phase 2 reads dP, forms dS = p (dP - D) and
+// writes it (bf16) over the columns of dP it has just read.  Warp 8 lane 0 issues the TMA loads,
+// warp 9 lane 0 issues every tcgen05.mma.
+// TMEM (512 columns), dQ kernel: S ping [0,128), S pong [128,256), dP/dS [256,384), dQ [384,384+d).
+//                     dK/dV kernel: S^T/P^T [0,128), dP^T/dS^T [128,256), dK [256,256+d), dV [256+d,256+2d).
 // Every mbarrier wait is bounded; on expiry the CTA raises a flag, drains and reports MKA_ERR_TIMEOUT.
 #include "tc_ptx.cuh"
 
@@ -30,10 +34,9 @@ namespace {
 
 constexpr int kThreads = 320;
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
-constexpr int kSub = 64;                              // rows of a streamed sub-tile
-constexpr uint32_t kPanel128 = 128 * 128;             // bytes of a [128 rows][64 bf16] panel
-constexpr uint32_t kPanel64 = 64 * 128;               // bytes of a [64 rows][64 bf16] panel
-constexpr int kMaxStages = 8;
+constexpr int kBlk = 128;                             // rows of every tile
+constexpr uint32_t kPanel = 128 * 128;                // bytes of a [128 rows][64 bf16] panel
+constexpr int kMaxStages = 4;
 
 struct BwdMaps {
     CUtensorMap q, dO;
@@ -56,23 +59,24 @@ struct BwdTcParams {
 template <int DH>
 struct BCfg {
     static constexpr int kPanels = DH / 64;
-    static constexpr uint32_t kBig = kPanels * kPanel128;     // a 128-row tile
-    static constexpr uint32_t kSmall = kPanels * kPanel64;    // a 64-row sub-tile
-    static constexpr int kStages = DH == 128 ? 4 : 8;         // also keeps the CTA above half of shared memory
-    static constexpr uint32_t kStatBytes = kSub * sizeof(float2);
-    static constexpr uint32_t kSmemDq = 2 * kBig + kStages * 2 * kSmall + 1024;
-    static constexpr uint32_t kSmemDkv = 2 * kBig + kStages * (2 * kSmall + kStatBytes) + 1024;
+    static constexpr uint32_t kTile = kPanels * kPanel;       // a 128-row tile
+    static constexpr int kStages = DH == 128 ? 2 : 4;         // also keeps the CTA above half of shared memory
+    static constexpr uint32_t kStatBytes = kBlk * sizeof(float2);
+    static constexpr uint32_t kSmemDq = 2 * kTile + kStages * 2 * kTile + 1024;
+    static constexpr uint32_t kSmemDkv = 2 * kTile + kStages * (2 * kTile + kStatBytes) + 1024;
     // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
-    static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSub >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlk >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     static constexpr uint32_t kIdescAcc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-    static constexpr uint32_t kAccCol = 256;                  // first accumulator column
 };
 
 struct BwdBarriers {
     uint64_t fixed_full;                                  // the CTA's own (non-streamed) tiles
-    uint64_t a_full[kMaxStages], a_empty[kMaxStages];     // streamed operand ring (first stream)
-    uint64_t b_full[kMaxStages], b_empty[kMaxStages];     // streamed operand ring (second stream; dQ kernel only)
-    uint64_t sdp_full[2], ds_full[2];
+    uint64_t a_full[kMaxStages], a_empty[kMaxStages];     // streamed ring (dQ kernel: K tiles; dK/dV kernel: Q + dO + stats)
+    uint64_t b_full[kMaxStages], b_empty[kMaxStages];     // second streamed ring (dQ kernel: V tiles)
+    uint64_t s_full[2];                                   // S landed in TMEM (dQ kernel: ping, pong)
+    uint64_t dp_full;                                     // dP landed in TMEM
+    uint64_t p_full;                                      // phase 1 done (dK/dV kernel: P^T written)
+    uint64_t ds_full;                                     // phase 2 done: dS written
     uint64_t acc_done;
 };
 
@@ -121,16 +125,16 @@ __global__ void __launch_bounds__(256) bwd_prep_kernel(const __nv_bfloat16* __re
     if (lane == 0) { s0[r] = o0; s1[r] = o1; s2[r] = o2; }
 }
 
-// Key sub-tile range [first, end) (64-row units) of query rows [r0, r1] on one level.
-__device__ __forceinline__ void sub_range(int level, long long r0, long long r1, int q_offset, int window, long long n,
-                                          int& first, int& end) {
+// Key tile range [first, end) (128-row units) of query rows [r0, r1] on one level.
+__device__ __forceinline__ void key_tile_range(int level, long long r0, long long r1, int q_offset, int window, long long n,
+                                               int& first, int& end) {
     long long lo_f, hi_f, lo_l, hi_l;
     visible_range(level, r0 + q_offset, window, n, 0, lo_f, hi_f);
     visible_range(level, r1 + q_offset, window, n, 0, lo_l, hi_l);
     const long long hi = hi_l > hi_f ? hi_l : hi_f;
     if (hi <= lo_f) { first = end = 0; return; }
-    first = (int)(lo_f / kSub);
-    end = (int)((hi + kSub - 1) / kSub);
+    first = (int)(lo_f / kBlk);
+    end = (int)((hi + kBlk - 1) / kBlk);
 }
 
 __device__ __forceinline__ void store_row_bf16(__nv_bfloat16* dst, const uint32_t (&o)[32], float mul) {
@@ -145,16 +149,21 @@ __device__ __forceinline__ void store_row_bf16(__nv_bfloat16* dst, const uint32_
     }
 }
 
+// A-operand column (32-bit TMEM columns) of K-step k of a 128-wide bf16 row that the two warpgroups wrote
+// as two packed halves: keys 0-63 at columns [0,32), keys 64-127 at columns [64,96) of the region.
+__device__ __forceinline__ uint32_t packed_half_col(int k) { return (uint32_t)((k >> 2) * 64 + (k & 3) * 8); }
+
 // ------------------------------------------------------------------------------------------ dQ
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdTcParams p) {
     using C = BCfg<DH>;
+    constexpr uint32_t kColS = 0, kColDP = 256, kColAcc = 384;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* sQ = smem;
-    uint8_t* sdO = sQ + C::kBig;
-    uint8_t* sK = sdO + C::kBig;                          // kStages sub-tiles
-    uint8_t* sV = sK + C::kStages * C::kSmall;            // kStages sub-tiles
+    uint8_t* sdO = sQ + C::kTile;
+    uint8_t* sK = sdO + C::kTile;                         // kStages tiles
+    uint8_t* sV = sK + C::kStages * C::kTile;             // kStages tiles
     __shared__ BwdBarriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -164,8 +173,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
     const int b = blockIdx.z, h = blockIdx.y;
     const long long bh = (long long)b * p.H + h;
     const int qtile = gridDim.x - 1 - blockIdx.x;          // latest (heaviest) rows first
-    const long long m0 = (long long)qtile * 128;
-    const long long m_last = (m0 + 127 < p.T - 1) ? m0 + 127 : p.T - 1;
+    const long long m0 = (long long)qtile * kBlk;
+    const long long m_last = (m0 + kBlk - 1 < p.T - 1) ? m0 + kBlk - 1 : p.T - 1;
 
     if (tid == 0) {
         abort_flag = 0;
@@ -174,7 +183,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
             mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1);
             mbar_init(&bar.b_full[s], 1); mbar_init(&bar.b_empty[s], 1);
         }
-        for (int w = 0; w < 2; ++w) { mbar_init(&bar.sdp_full[w], 1); mbar_init(&bar.ds_full[w], 128); }
+        mbar_init(&bar.s_full[0], 1); mbar_init(&bar.s_full[1], 1);
+        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 256); mbar_init(&bar.ds_full, 256);
         mbar_init(&bar.acc_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -191,18 +201,18 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
     int first[3], end[3];
 #pragma unroll
     for (int l = 0; l < 3; ++l) {
-        if (p.n[l] > 0) sub_range(l, m0, m_last, p.q_offset, p.window, p.n[l], first[l], end[l]);
+        if (p.n[l] > 0) key_tile_range(l, m0, m_last, p.q_offset, p.window, p.n[l], first[l], end[l]);
         else first[l] = end[l] = 0;
     }
     const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
 
     if (warp == kProducerWarp) {
         if (lane == 0) {
-            mbar_expect_tx(&bar.fixed_full, 2 * C::kBig);
+            mbar_expect_tx(&bar.fixed_full, 2 * C::kTile);
 #pragma unroll
             for (int pn = 0; pn < C::kPanels; ++pn) {
-                tma_load_4d(sQ + pn * kPanel128, &maps.q, pn * 64, (int)m0, h, b, &bar.fixed_full);
-                tma_load_4d(sdO + pn * kPanel128, &maps.dO, pn * 64, (int)m0, h, b, &bar.fixed_full);
+                tma_load_4d(sQ + pn * kPanel, &maps.q, pn * 64, (int)m0, h, b, &bar.fixed_full);
+                tma_load_4d(sdO + pn * kPanel, &maps.dO, pn * 64, (int)m0, h, b, &bar.fixed_full);
             }
             int issued_k = 0, issued_v = 0;
             bool ok = true;
@@ -211,16 +221,16 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                     const int s = issued_k % C::kStages;
                     const uint32_t ph = (uint32_t)(issued_k / C::kStages) & 1u;
                     if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
-                    mbar_expect_tx(&bar.a_full[s], C::kSmall);
+                    mbar_expect_tx(&bar.a_full[s], C::kTile);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sK + s * C::kSmall + pn * kPanel64, &maps.k[l], pn * 64, kt * kSub, h, b, &bar.a_full[s]);
+                        tma_load_4d(sK + s * C::kTile + pn * kPanel, &maps.k[l], pn * 64, kt * kBlk, h, b, &bar.a_full[s]);
                     ++issued_k;
                     if (!mbar_wait(&bar.b_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
-                    mbar_expect_tx(&bar.b_full[s], C::kSmall);
+                    mbar_expect_tx(&bar.b_full[s], C::kTile);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sV + s * C::kSmall + pn * kPanel64, &maps.v[l], pn * 64, kt * kSub, h, b, &bar.b_full[s]);
+                        tma_load_4d(sV + s * C::kTile + pn * kPanel, &maps.v[l], pn * 64, kt * kBlk, h, b, &bar.b_full[s]);
                     ++issued_v;
                 }
             }
@@ -232,50 +242,55 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 mbar_wait(&bar.b_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
     } else if (warp == kMmaWarp) {
-        if (lane == 0) {
+        if (lane == 0 && E > 0) {
             bool ok = mbar_wait(&bar.fixed_full, 0, abortp);
             tc_fence_after();
             const uint32_t q_addr = smem_u32(sQ), g_addr = smem_u32(sdO), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-            auto issue_dq = [&](int e) -> bool {           // dQ += dS(e) K(e)
-                const int w = e & 1, s = e % C::kStages;
-                if (!mbar_wait(&bar.ds_full[w], (uint32_t)(e >> 1) & 1u, abortp)) return false;
+            auto issue_s = [&](int e) -> bool {             // S(e) = Q K(e)^T into the ping/pong buffer e & 1
+                const int s = e % C::kStages;
+                if (!mbar_wait(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
                 tc_fence_after();
-                const uint32_t ka = k_addr + s * C::kSmall;
+                const uint32_t ka = k_addr + s * C::kTile;
 #pragma unroll
-                for (int k = 0; k < kSub / 16; ++k)
-                    mma_ts(tmem + C::kAccCol, tmem + w * 128 + k * 8, desc_mnmajor(ka + k * 2048, kPanel64), C::kIdescAcc,
-                           (e > 0 || k > 0) ? 1u : 0u);
-                mma_commit(&bar.a_empty[s]);
+                for (int k = 0; k < DH / 16; ++k) {
+                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
+                    mma_ss(tmem + kColS + (e & 1) * 128, desc_kmajor(q_addr + off), desc_kmajor(ka + off), C::kIdescS, k > 0);
+                }
+                mma_commit(&bar.s_full[e & 1]);
                 return true;
             };
+            if (ok) ok = issue_s(0);
             for (int e = 0; e < E && ok; ++e) {
-                const int w = e & 1, s = e % C::kStages;
-                const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
-                if (!mbar_wait(&bar.a_full[s], ph, abortp) || !mbar_wait(&bar.b_full[s], ph, abortp)) { ok = false; break; }
+                const int s = e % C::kStages;
+                if (!mbar_wait(&bar.b_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t ka = k_addr + s * C::kSmall, va = v_addr + s * C::kSmall;
+                const uint32_t ka = k_addr + s * C::kTile, va = v_addr + s * C::kTile;
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k)          // S = Q K^T
-                    mma_ss(tmem + w * 128, desc_kmajor(q_addr + (k / 4) * kPanel128 + (k % 4) * 32),
-                           desc_kmajor(ka + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
-#pragma unroll
-                for (int k = 0; k < DH / 16; ++k)          // dP = dO V^T
-                    mma_ss(tmem + w * 128 + 64, desc_kmajor(g_addr + (k / 4) * kPanel128 + (k % 4) * 32),
-                           desc_kmajor(va + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
-                mma_commit(&bar.sdp_full[w]);
+                for (int k = 0; k < DH / 16; ++k) {        // dP(e) = dO V(e)^T  (dS(e-1), which shares the columns, was consumed by dQ(e-1) issued before)
+                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
+                    mma_ss(tmem + kColDP, desc_kmajor(g_addr + off), desc_kmajor(va + off), C::kIdescS, k > 0);
+                }
+                mma_commit(&bar.dp_full);
                 mma_commit(&bar.b_empty[s]);
-                if (e > 0 && !issue_dq(e - 1)) { ok = false; break; }
+                if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
+                if (!mbar_wait(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < kBlk / 16; ++k)         // dQ += dS(e) K(e)
+                    mma_ts(tmem + kColAcc, tmem + kColDP + packed_half_col(k), desc_mnmajor(ka + k * 2048, kPanel), C::kIdescAcc,
+                           (e > 0 || k > 0) ? 1u : 0u);
+                mma_commit(&bar.a_empty[s]);
             }
-            if (ok && E > 0 && issue_dq(E - 1)) mma_commit(&bar.acc_done);
+            if (ok) mma_commit(&bar.acc_done);
         }
     } else {
-        // ------------------------------------------------------------ softmax warpgroups
+        // ------------------------------------------------------------ element-wise warpgroups (thread = query row, 64 of the 128 columns)
         const int w = warp >> 2;
         const int r = tid & 127;
         const long long t = m0 + r;
         const bool row_valid = t < p.T;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t st_addr = tmem + lane_base + w * 128;
+        const uint32_t dp_addr = tmem + lane_base + kColDP + w * 64;
         float Dt = 0.f, bias[3] = {-INFINITY, -INFINITY, -INFINITY};
         if (row_valid) {
 #pragma unroll
@@ -285,7 +300,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 bias[l] = sv.y;
             }
         }
-        float Al[3] = {0.f, 0.f, 0.f}, Sl[3] = {0.f, 0.f, 0.f};   // per level: sum p dP and sum p
+        float Al[3] = {0.f, 0.f, 0.f}, Sl[3] = {0.f, 0.f, 0.f};   // per level: sum p dP and sum p over this thread's columns
         bool ok = true;
         int e = 0;
 #pragma unroll
@@ -298,46 +313,60 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 long long lo_f, hi_f, lo_l, hi_l;
                 visible_range(l, m0 + p.q_offset, p.window, p.n[l], 0, lo_f, hi_f);
                 visible_range(l, m_last + p.q_offset, p.window, p.n[l], 0, lo_l, hi_l);
-                full_first = (int)((lo_l + kSub - 1) / kSub);
-                full_end = (int)(hi_f / kSub);
-                if (m_last - m0 + 1 < 128) full_end = full_first;           // ragged query tile: always mask
+                full_first = (int)((lo_l + kBlk - 1) / kBlk);
+                full_end = (int)(hi_f / kBlk);
+                if (m_last - m0 + 1 < kBlk) full_end = full_first;          // ragged query tile: always mask
             }
             float a0 = 0.f, a1 = 0.f, z0 = 0.f, z1 = 0.f;
+            const float bl = bias[l];
             for (int kt = first[l]; kt < end[l]; ++kt, ++e) {
-                if ((e & 1) != w) continue;
-                ok = mbar_wait(&bar.sdp_full[w], (uint32_t)(e >> 1) & 1u, abortp);
+                // phase 1: p = 2^(s * scale + bias) for this thread's 64 columns (needs S only)
+                ok = mbar_wait(&bar.s_full[e & 1], (uint32_t)(e >> 1) & 1u, abortp);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                float s[kSub], dp[kSub];
-                tmem_ld32(st_addr, reinterpret_cast<uint32_t*>(s));
-                tmem_ld32(st_addr + 32, reinterpret_cast<uint32_t*>(s) + 32);
-                tmem_ld32(st_addr + 64, reinterpret_cast<uint32_t*>(dp));
-                tmem_ld32(st_addr + 96, reinterpret_cast<uint32_t*>(dp) + 32);
-                tmem_ld_wait();
+                float pr[64];
+                {
+                    const uint32_t s_addr = tmem + lane_base + kColS + (e & 1) * 128 + w * 64;
+                    tmem_ld32(s_addr, reinterpret_cast<uint32_t*>(pr));
+                    tmem_ld32(s_addr + 32, reinterpret_cast<uint32_t*>(pr) + 32);
+                    tmem_ld_wait();
+                }
                 if (!(kt >= full_first && kt < full_end)) {
-                    const int c_lo = (int)max(-1LL, min(lo - (long long)kt * kSub, (long long)kSub));
-                    const int c_hi = (int)max(-1LL, min(hi - (long long)kt * kSub, (long long)kSub));
+                    const long long j0 = (long long)kt * kBlk + w * 64;
+                    const int c_lo = (int)max(-1LL, min(lo - j0, 64LL));
+                    const int c_hi = (int)max(-1LL, min(hi - j0, 64LL));
 #pragma unroll
-                    for (int c = 0; c < kSub; ++c)
-                        if (c < c_lo || c >= c_hi) s[c] = -INFINITY;
+                    for (int c = 0; c < 64; ++c)
+                        if (c < c_lo || c >= c_hi) pr[c] = -INFINITY;
                 }
-                uint32_t pk[kSub / 2];
-                const float bl = bias[l];
 #pragma unroll
-                for (int c = 0; c < kSub; c += 2) {
-                    const float p0 = ex2(fmaf(s[c], p.scale_log2, bl));
-                    const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, bl));
-                    a0 = fmaf(p0, dp[c], a0);
-                    a1 = fmaf(p1, dp[c + 1], a1);
-                    z0 += p0;
-                    z1 += p1;
-                    pk[c / 2] = pack_bf16(p0 * (dp[c] - Dt), p1 * (dp[c + 1] - Dt));
+                for (int c = 0; c < 64; c += 2) {
+                    pr[c] = ex2(fmaf(pr[c], p.scale_log2, bl));
+                    pr[c + 1] = ex2(fmaf(pr[c + 1], p.scale_log2, bl));
+                    z0 += pr[c];
+                    z1 += pr[c + 1];
                 }
-                tmem_st32(st_addr, pk);
+                // phase 2: dS = p (dP - D), written (bf16) over the dP columns just read
+                ok = mbar_wait(&bar.dp_full, (uint32_t)e & 1u, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                float dp[64];
+                tmem_ld32(dp_addr, reinterpret_cast<uint32_t*>(dp));
+                tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(dp) + 32);
+                tmem_ld_wait();
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 64; c += 2) {
+                    a0 = fmaf(pr[c], dp[c], a0);
+                    a1 = fmaf(pr[c + 1], dp[c + 1], a1);
+                    pk[c / 2] = pack_bf16(pr[c] * (dp[c] - Dt), pr[c + 1] * (dp[c + 1] - Dt));
+                }
+                tmem_st32(dp_addr, pk);
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(&bar.ds_full[w]);
+                mbar_arrive(&bar.ds_full);
             }
             Al[l] = a0 + a1;
             Sl[l] = z0 + z1;
@@ -354,7 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
             for (int c0 = w * (DH / 2); c0 < (w + 1) * (DH / 2); c0 += 32) {
                 uint32_t o[32];
                 if (E > 0) {
-                    tmem_ld32(tmem + lane_base + C::kAccCol + c0, o);
+                    tmem_ld32(tmem + lane_base + kColAcc + c0, o);
                     tmem_ld_wait();
                 } else {
 #pragma unroll
@@ -365,7 +394,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
         }
         // Gate-logit gradient of this head: G_l = sum_{j in l} p (dP - D').  D' = sum p dP / sum p equals
         // dO . O in exact arithmetic but does not inherit the rounding of O to bf16, so sum_l G_l = 0 holds
-        // to fp32 accuracy.  The two warpgroups hold disjoint sub-tiles: add their partial sums first.
+        // to fp32 accuracy.  The two warpgroups hold disjoint columns: add their partial sums first.
         if (w == 1) {
 #pragma unroll
             for (int l = 0; l < 3; ++l) { gsm[r][l] = Al[l]; gsm[r][3 + l] = Sl[l]; }
@@ -393,13 +422,14 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdTcParams p) {
     using C = BCfg<DH>;
+    constexpr uint32_t kColS = 0, kColDP = 128, kColDK = 256, kColDV = 256 + DH;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* sK = smem;
-    uint8_t* sV = sK + C::kBig;
-    uint8_t* sQ = sV + C::kBig;                           // kStages sub-tiles
-    uint8_t* sdO = sQ + C::kStages * C::kSmall;           // kStages sub-tiles
-    float2* sStat = reinterpret_cast<float2*>(sdO + C::kStages * C::kSmall);   // kStages x 64
+    uint8_t* sV = sK + C::kTile;
+    uint8_t* sQ = sV + C::kTile;                          // kStages tiles
+    uint8_t* sdO = sQ + C::kStages * C::kTile;            // kStages tiles
+    float2* sStat = reinterpret_cast<float2*>(sdO + C::kStages * C::kTile);   // kStages x 128
     __shared__ BwdBarriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -416,22 +446,23 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
         else { lvl = 0; kt = x - p.kv_tiles[2] - p.kv_tiles[1]; }
     }
     const long long n = p.n[lvl];
-    const long long j0 = (long long)kt * 128;
-    const long long j_last = (j0 + 127 < n - 1) ? j0 + 127 : n - 1;
+    const long long j0 = (long long)kt * kBlk;
+    const long long j_last = (j0 + kBlk - 1 < n - 1) ? j0 + kBlk - 1 : n - 1;
     // queries t (position t + q_offset) that can see a key of this tile
     long long t_lo = 0, t_hi = p.T;
     if (lvl == 0) { t_lo = j0 - p.q_offset; t_hi = j_last + p.window - p.q_offset; }
     else if (lvl == 1) { t_lo = j0 - p.q_offset; }
     if (t_lo < 0) t_lo = 0;
     if (t_hi > p.T) t_hi = p.T;
-    const int first = t_hi > t_lo ? (int)(t_lo / kSub) : 0;
-    const int E = t_hi > t_lo ? (int)((t_hi + kSub - 1) / kSub) - first : 0;
+    const int first = t_hi > t_lo ? (int)(t_lo / kBlk) : 0;
+    const int E = t_hi > t_lo ? (int)((t_hi + kBlk - 1) / kBlk) - first : 0;
 
     if (tid == 0) {
         abort_flag = 0;
         mbar_init(&bar.fixed_full, 1);
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1); }
-        for (int w = 0; w < 2; ++w) { mbar_init(&bar.sdp_full[w], 1); mbar_init(&bar.ds_full[w], 128); }
+        mbar_init(&bar.s_full[0], 1);
+        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 256); mbar_init(&bar.ds_full, 256);
         mbar_init(&bar.acc_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -446,132 +477,155 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     volatile int* abortp = &abort_flag;
 
     if (warp == kProducerWarp) {
-        if (lane == 0) {
-            bool ok = true;
+        if (lane == 0 && E > 0) {
             int issued = 0;
-            if (E > 0) {
-                mbar_expect_tx(&bar.fixed_full, 2 * C::kBig);
+            mbar_expect_tx(&bar.fixed_full, 2 * C::kTile);
+#pragma unroll
+            for (int pn = 0; pn < C::kPanels; ++pn) {
+                tma_load_4d(sK + pn * kPanel, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                tma_load_4d(sV + pn * kPanel, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+            }
+            const float2* stat = p.stats[lvl] + bh * p.Tpad;
+            for (int e = 0; e < E; ++e) {
+                const int s = e % C::kStages;
+                const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) break;
+                const int tt = (first + e) * kBlk;
+                mbar_expect_tx(&bar.a_full[s], 2 * C::kTile + C::kStatBytes);
 #pragma unroll
                 for (int pn = 0; pn < C::kPanels; ++pn) {
-                    tma_load_4d(sK + pn * kPanel128, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
-                    tma_load_4d(sV + pn * kPanel128, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                    tma_load_4d(sQ + s * C::kTile + pn * kPanel, &maps.q, pn * 64, tt, h, b, &bar.a_full[s]);
+                    tma_load_4d(sdO + s * C::kTile + pn * kPanel, &maps.dO, pn * 64, tt, h, b, &bar.a_full[s]);
                 }
-                const float2* stat = p.stats[lvl] + bh * p.Tpad;
-                for (int e = 0; e < E; ++e) {
-                    const int s = e % C::kStages;
-                    const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
-                    if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
-                    const int tt = (first + e) * kSub;
-                    mbar_expect_tx(&bar.a_full[s], 2 * C::kSmall + C::kStatBytes);
-#pragma unroll
-                    for (int pn = 0; pn < C::kPanels; ++pn) {
-                        tma_load_4d(sQ + s * C::kSmall + pn * kPanel64, &maps.q, pn * 64, tt, h, b, &bar.a_full[s]);
-                        tma_load_4d(sdO + s * C::kSmall + pn * kPanel64, &maps.dO, pn * 64, tt, h, b, &bar.a_full[s]);
-                    }
-                    bulk_load(sStat + s * kSub, stat + tt, C::kStatBytes, &bar.a_full[s]);
-                    ++issued;
-                }
-                mbar_wait(&bar.fixed_full, 0, abortp);
-                for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
-                    mbar_wait(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+                bulk_load(sStat + s * kBlk, stat + tt, C::kStatBytes, &bar.a_full[s]);
+                ++issued;
             }
-            (void)ok;
+            mbar_wait(&bar.fixed_full, 0, abortp);
+            for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
+                mbar_wait(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
     } else if (warp == kMmaWarp) {
         if (lane == 0 && E > 0) {
             bool ok = mbar_wait(&bar.fixed_full, 0, abortp);
             tc_fence_after();
             const uint32_t k_addr = smem_u32(sK), v_addr = smem_u32(sV), q_addr = smem_u32(sQ), g_addr = smem_u32(sdO);
-            auto issue_acc = [&](int e) -> bool {          // dV += P^T(e) dO(e);  dK += dS^T(e) Q(e)
-                const int w = e & 1, s = e % C::kStages;
-                if (!mbar_wait(&bar.ds_full[w], (uint32_t)(e >> 1) & 1u, abortp)) return false;
+            auto issue_s = [&](int e) -> bool {             // S^T(e) = K Q(e)^T   (P^T(e-1), which shares the columns, was consumed by dV(e-1) issued before)
+                const int s = e % C::kStages;
+                if (!mbar_wait(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
                 tc_fence_after();
-                const uint32_t qa = q_addr + s * C::kSmall, ga = g_addr + s * C::kSmall;
+                const uint32_t qa = q_addr + s * C::kTile;
 #pragma unroll
-                for (int k = 0; k < kSub / 16; ++k)
-                    mma_ts(tmem + C::kAccCol + DH, tmem + w * 128 + k * 8, desc_mnmajor(ga + k * 2048, kPanel64), C::kIdescAcc,
-                           (e > 0 || k > 0) ? 1u : 0u);
-#pragma unroll
-                for (int k = 0; k < kSub / 16; ++k)
-                    mma_ts(tmem + C::kAccCol, tmem + w * 128 + 64 + k * 8, desc_mnmajor(qa + k * 2048, kPanel64), C::kIdescAcc,
-                           (e > 0 || k > 0) ? 1u : 0u);
-                mma_commit(&bar.a_empty[s]);
+                for (int k = 0; k < DH / 16; ++k) {
+                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
+                    mma_ss(tmem + kColS, desc_kmajor(k_addr + off), desc_kmajor(qa + off), C::kIdescS, k > 0);
+                }
+                mma_commit(&bar.s_full[0]);
                 return true;
             };
+            auto issue_dp = [&](int e) {                    // dP^T(e) = V dO(e)^T  (its stage was awaited by issue_s(e))
+                const uint32_t ga = g_addr + (e % C::kStages) * C::kTile;
+#pragma unroll
+                for (int k = 0; k < DH / 16; ++k) {
+                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
+                    mma_ss(tmem + kColDP, desc_kmajor(v_addr + off), desc_kmajor(ga + off), C::kIdescS, k > 0);
+                }
+                mma_commit(&bar.dp_full);
+            };
+            if (ok) ok = issue_s(0);
+            if (ok) issue_dp(0);
             for (int e = 0; e < E && ok; ++e) {
-                const int w = e & 1, s = e % C::kStages;
-                const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
-                if (!mbar_wait(&bar.a_full[s], ph, abortp)) { ok = false; break; }
+                const int s = e % C::kStages;
+                const uint32_t qa = q_addr + s * C::kTile, ga = g_addr + s * C::kTile;
+                if (!mbar_wait(&bar.p_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t qa = q_addr + s * C::kSmall, ga = g_addr + s * C::kSmall;
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k)          // S^T = K Q^T
-                    mma_ss(tmem + w * 128, desc_kmajor(k_addr + (k / 4) * kPanel128 + (k % 4) * 32),
-                           desc_kmajor(qa + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
+                for (int k = 0; k < kBlk / 16; ++k)         // dV += P^T(e) dO(e)
+                    mma_ts(tmem + kColDV, tmem + kColS + packed_half_col(k), desc_mnmajor(ga + k * 2048, kPanel), C::kIdescAcc,
+                           (e > 0 || k > 0) ? 1u : 0u);
+                if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
+                if (!mbar_wait(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k)          // dP^T = V dO^T
-                    mma_ss(tmem + w * 128 + 64, desc_kmajor(v_addr + (k / 4) * kPanel128 + (k % 4) * 32),
-                           desc_kmajor(ga + (k / 4) * kPanel64 + (k % 4) * 32), C::kIdescS, k > 0);
-                mma_commit(&bar.sdp_full[w]);
-                if (e > 0 && !issue_acc(e - 1)) { ok = false; break; }
+                for (int k = 0; k < kBlk / 16; ++k)         // dK += dS^T(e) Q(e)
+                    mma_ts(tmem + kColDK, tmem + kColDP + packed_half_col(k), desc_mnmajor(qa + k * 2048, kPanel), C::kIdescAcc,
+                           (e > 0 || k > 0) ? 1u : 0u);
+                mma_commit(&bar.a_empty[s]);
+                if (e + 1 < E) issue_dp(e + 1);
             }
-            if (ok && issue_acc(E - 1)) mma_commit(&bar.acc_done);
+            if (ok) mma_commit(&bar.acc_done);
         }
     } else {
-        // ------------------------------------------------------------ softmax warpgroups (thread = key row)
+        // ------------------------------------------------------------ element-wise warpgroups (thread = key row, 64 of the 128 query columns)
         const int w = warp >> 2;
         const int r = tid & 127;
         const long long j = j0 + r;
         const bool row_valid = j < n;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t st_addr = tmem + lane_base + w * 128;
+        const uint32_t s_addr = tmem + lane_base + kColS + w * 64;
+        const uint32_t dp_addr = tmem + lane_base + kColDP + w * 64;
         // queries [q_lo, q_hi) that see key j (the bound t < T is carried by the padded biases)
         long long q_lo = 0, q_hi = 0;
         if (row_valid) {
             q_lo = lvl == 2 ? 0 : j - p.q_offset;
             q_hi = lvl == 0 ? j + p.window - p.q_offset : (long long)p.Tpad;
         }
-        // sub-tiles whose every (key, query) pair is visible need no mask
-        const bool rows_full = j0 + 127 < n;
+        const bool rows_full = j0 + kBlk - 1 < n;
         bool ok = true;
-        for (int e = w; e < E; e += 2) {
+        for (int e = 0; e < E; ++e) {
             const int s = e % C::kStages;
-            const long long tt = (long long)(first + e) * kSub;
-            ok = mbar_wait(&bar.sdp_full[w], (uint32_t)(e >> 1) & 1u, abortp);
+            const long long tt = (long long)(first + e) * kBlk;        // first query of the tile
+            const float4* stat = reinterpret_cast<const float4*>(sStat + s * kBlk + w * 64);   // {D, bias} of two queries per load
+            // phase 1: P^T = 2^(s * scale + bias_t) for this thread's 64 query columns
+            ok = mbar_wait(&bar.s_full[0], (uint32_t)e & 1u, abortp);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            float sc[kSub], dp[kSub];
-            tmem_ld32(st_addr, reinterpret_cast<uint32_t*>(sc));
-            tmem_ld32(st_addr + 32, reinterpret_cast<uint32_t*>(sc) + 32);
-            tmem_ld32(st_addr + 64, reinterpret_cast<uint32_t*>(dp));
-            tmem_ld32(st_addr + 96, reinterpret_cast<uint32_t*>(dp) + 32);
+            float pr[64];
+            tmem_ld32(s_addr, reinterpret_cast<uint32_t*>(pr));
+            tmem_ld32(s_addr + 32, reinterpret_cast<uint32_t*>(pr) + 32);
             tmem_ld_wait();
+            // tiles whose every (key, query) pair is visible need no mask
             bool full = rows_full;
             if (lvl != 2) full = full && (j_last - p.q_offset <= tt);
-            if (lvl == 0) full = full && (j0 + p.window - p.q_offset >= tt + kSub);
+            if (lvl == 0) full = full && (j0 + p.window - p.q_offset >= tt + kBlk);
             if (!full) {
-                const int c_lo = (int)max(-1LL, min(q_lo - tt, (long long)kSub));
-                const int c_hi = (int)max(-1LL, min(q_hi - tt, (long long)kSub));
+                const long long c0 = tt + w * 64;
+                const int c_lo = (int)max(-1LL, min(q_lo - c0, 64LL));
+                const int c_hi = (int)max(-1LL, min(q_hi - c0, 64LL));
 #pragma unroll
-                for (int c = 0; c < kSub; ++c)
-                    if (c < c_lo || c >= c_hi) sc[c] = -INFINITY;
+                for (int c = 0; c < 64; ++c)
+                    if (c < c_lo || c >= c_hi) pr[c] = -INFINITY;
             }
-            const float4* stat = reinterpret_cast<const float4*>(sStat + s * kSub);   // two queries per load
-            uint32_t pkP[kSub / 2], pkD[kSub / 2];
+            uint32_t pk[32];
 #pragma unroll
-            for (int c = 0; c < kSub; c += 2) {
-                const float4 sv = stat[c / 2];                                          // {D_c, bias_c, D_c+1, bias_c+1}
-                const float p0 = ex2(fmaf(sc[c], p.scale_log2, sv.y));
-                const float p1 = ex2(fmaf(sc[c + 1], p.scale_log2, sv.w));
-                pkP[c / 2] = pack_bf16(p0, p1);
-                pkD[c / 2] = pack_bf16(p0 * (dp[c] - sv.x), p1 * (dp[c + 1] - sv.z));
+            for (int c = 0; c < 64; c += 2) {
+                const float4 sv = stat[c / 2];
+                pr[c] = ex2(fmaf(pr[c], p.scale_log2, sv.y));
+                pr[c + 1] = ex2(fmaf(pr[c + 1], p.scale_log2, sv.w));
+                pk[c / 2] = pack_bf16(pr[c], pr[c + 1]);
             }
-            tmem_st32(st_addr, pkP);
-            tmem_st32(st_addr + 64, pkD);
+            tmem_st32(s_addr, pk);
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(&bar.ds_full[w]);
+            mbar_arrive(&bar.p_full);
+            // phase 2: dS^T = P^T (dP^T - D_t), written over the dP^T columns just read
+            ok = mbar_wait(&bar.dp_full, (uint32_t)e & 1u, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float dp[64];
+            tmem_ld32(dp_addr, reinterpret_cast<uint32_t*>(dp));
+            tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(dp) + 32);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 64; c += 2) {
+                const float4 sv = stat[c / 2];
+                pk[c / 2] = pack_bf16(pr[c] * (dp[c] - sv.x), pr[c + 1] * (dp[c + 1] - sv.z));
+            }
+            tmem_st32(dp_addr, pk);
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(&bar.ds_full);
         }
         // ------------------------------------------------------------ epilogue: warpgroup 0 writes dK, 1 writes dV
         if (ok && E > 0) {
@@ -587,7 +641,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             for (int c0 = 0; c0 < DH; c0 += 32) {
                 uint32_t o[32];
                 if (E > 0) {
-                    tmem_ld32(tmem + lane_base + C::kAccCol + w * DH + c0, o);
+                    tmem_ld32(tmem + lane_base + (w == 0 ? kColDK : kColDV) + c0, o);
                     tmem_ld_wait();
                 } else {
 #pragma unroll
@@ -607,7 +661,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
 template <int DH>
 cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_t st) {
     using C = BCfg<DH>;
-    const int Tpad = (bp.T + kSub - 1) / kSub * kSub;
+    const int Tpad = (bp.T + kBlk - 1) / kBlk * kBlk;
     const long long rows_pad = (long long)bp.B * bp.H * Tpad;
     float2* stats[3];
     for (int l = 0; l < 3; ++l) stats[l] = reinterpret_cast<float2*>(bp.stats) + (long long)l * rows_pad;
@@ -633,7 +687,7 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
     p.scale = bp.scale; p.scale_log2 = bp.scale * kLog2e;
     p.status = status_word;
 
-    // dQ: 128-row Q / dO tiles, 64-row key sub-tiles
+    // both kernels move 128-row tiles (box = 64 columns x 128 rows)
     {
         BwdMaps m;
         if (!make_bf16_map(&m.q, bp.Q, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, 128) ||
@@ -641,8 +695,8 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
             return cudaErrorNotSupported;
         for (int l = 0; l < 3; ++l) {
             if (bp.L[l].n == 0) { m.k[l] = m.q; m.v[l] = m.q; continue; }
-            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kSub) ||
-                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kSub))
+            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kBlk) ||
+                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kBlk))
                 return cudaErrorNotSupported;
         }
         e = cudaFuncSetAttribute(bwd_dq_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemDq);
@@ -651,12 +705,11 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
         bwd_dq_tc_kernel<DH><<<grid, kThreads, C::kSmemDq, st>>>(m, p);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    // dK, dV: 128-row key tiles, 64-row Q / dO sub-tiles
     const int tiles = p.kv_tiles[0] + p.kv_tiles[1] + p.kv_tiles[2];
     if (tiles > 0) {
         BwdMaps m;
-        if (!make_bf16_map(&m.q, bp.Q, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, kSub) ||
-            !make_bf16_map(&m.dO, bp.dO, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, kSub))
+        if (!make_bf16_map(&m.q, bp.Q, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, kBlk) ||
+            !make_bf16_map(&m.dO, bp.dO, DH, bp.T, bp.H, bp.B, sq_n, sq_h, sq_b, kBlk))
             return cudaErrorNotSupported;
         for (int l = 0; l < 3; ++l) {
             if (bp.L[l].n == 0) { m.k[l] = m.q; m.v[l] = m.q; continue; }
