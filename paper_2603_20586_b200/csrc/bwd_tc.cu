@@ -22,8 +22,8 @@
 // warpgroup 0 takes columns 0-63 of a tile and warpgroup 1 columns 64-127.  Their work on a tile has
 // two phases so that it overlaps the tensor pipe: phase 1 needs only S (p = 2^(s*scale + bias), kept in
 // registers) and runs while dP is still being multiplied; phase 2 reads dP, forms dS = p (dP - D) and
-// writes it (bf16) over the columns of dP it has just read.  Warp 8 lane 0 issues the TMA loads,
-// warp 9 lane 0 issues every tcgen05.mma.
+// writes it (bf16) over the columns of dP it has just read.  Warp 8 lane 0 issues the TMA loads;
+// warp 9 issues every tcgen05.mma, running its loop converged with one elected lane issuing.
 // TMEM (512 columns), dQ kernel: S ping [0,128), S pong [128,256), dP/dS [256,384), dQ [384,384+d).
 //                     dK/dV kernel: S^T/P^T [0,128), dP^T/dS^T [128,256), dK [256,256+d), dV [256+d,256+2d).
 // Every mbarrier wait is bounded; on expiry the CTA raises a flag, drains and reports MKA_ERR_TIMEOUT.
@@ -62,7 +62,8 @@ struct BCfg {
     static constexpr uint32_t kTile = kPanels * kPanel;       // a 128-row tile
     static constexpr int kStages = DH == 128 ? 2 : 4;         // also keeps the CTA above half of shared memory
     static constexpr uint32_t kStatBytes = kBlk * sizeof(float2);
-    static constexpr uint32_t kSmemDq = 2 * kTile + kStages * 2 * kTile + 1024;
+    static constexpr int kStagesK = DH == 128 ? 3 : 4;        // K ring of the dQ kernel: K(e) stays in use until dQ(e), two tiles after it is first read
+    static constexpr uint32_t kSmemDq = 2 * kTile + (kStages + kStagesK) * kTile + 1024;
     static constexpr uint32_t kSmemDkv = 2 * kTile + kStages * (2 * kTile + kStatBytes) + 1024;
     // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
     static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlk >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -162,14 +163,15 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* sQ = smem;
     uint8_t* sdO = sQ + C::kTile;
-    uint8_t* sK = sdO + C::kTile;                         // kStages tiles
-    uint8_t* sV = sK + C::kStages * C::kTile;             // kStages tiles
+    uint8_t* sK = sdO + C::kTile;                         // kStagesK tiles
+    uint8_t* sV = sK + C::kStagesK * C::kTile;            // kStages tiles
+    float (*gsm)[6] = reinterpret_cast<float (*)[6]>(sQ); // epilogue scratch; Q is dead once the last S product has completed
     __shared__ BwdBarriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ float gsm[128][6];
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
     const int b = blockIdx.z, h = blockIdx.y;
     const long long bh = (long long)b * p.H + h;
     const int qtile = gridDim.x - 1 - blockIdx.x;          // latest (heaviest) rows first
@@ -218,70 +220,70 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
             bool ok = true;
             for (int l = 0; l < 3 && ok; ++l) {
                 for (int kt = first[l]; kt < end[l]; ++kt) {
-                    const int s = issued_k % C::kStages;
-                    const uint32_t ph = (uint32_t)(issued_k / C::kStages) & 1u;
+                    const int s = issued_k % C::kStagesK, sv = issued_k % C::kStages;
+                    const uint32_t ph = (uint32_t)(issued_k / C::kStagesK) & 1u, phv = (uint32_t)(issued_k / C::kStages) & 1u;
                     if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(&bar.a_full[s], C::kTile);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
                         tma_load_4d(sK + s * C::kTile + pn * kPanel, &maps.k[l], pn * 64, kt * kBlk, h, b, &bar.a_full[s]);
                     ++issued_k;
-                    if (!mbar_wait(&bar.b_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
-                    mbar_expect_tx(&bar.b_full[s], C::kTile);
+                    if (!mbar_wait(&bar.b_empty[sv], phv ^ 1u, abortp)) { ok = false; break; }
+                    mbar_expect_tx(&bar.b_full[sv], C::kTile);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sV + s * C::kTile + pn * kPanel, &maps.v[l], pn * 64, kt * kBlk, h, b, &bar.b_full[s]);
+                        tma_load_4d(sV + sv * C::kTile + pn * kPanel, &maps.v[l], pn * 64, kt * kBlk, h, b, &bar.b_full[sv]);
                     ++issued_v;
                 }
             }
             // every copy issued above must have landed before the shared memory can be given up
             mbar_wait(&bar.fixed_full, 0, abortp);
-            for (int i = issued_k > C::kStages ? issued_k - C::kStages : 0; i < issued_k; ++i)
-                mbar_wait(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+            for (int i = issued_k > C::kStagesK ? issued_k - C::kStagesK : 0; i < issued_k; ++i)
+                mbar_wait(&bar.a_full[i % C::kStagesK], (uint32_t)(i / C::kStagesK) & 1u, abortp);
             for (int i = issued_v > C::kStages ? issued_v - C::kStages : 0; i < issued_v; ++i)
                 mbar_wait(&bar.b_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
     } else if (warp == kMmaWarp) {
-        if (lane == 0 && E > 0) {
-            bool ok = mbar_wait(&bar.fixed_full, 0, abortp);
+        if (E > 0) {   // every lane runs the issue loop (converged); elect.sync inside the wrappers picks the issuing lane
+            bool ok = mbar_wait_warp(&bar.fixed_full, 0, abortp);
             tc_fence_after();
-            const uint32_t q_addr = smem_u32(sQ), g_addr = smem_u32(sdO), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+            // low descriptor words of the operands (see make_desc): K-major views for S and dP, MN-major view of K for dQ
+            const uint32_t q_lo = desc_lo_kmajor(smem_u32(sQ)), g_lo = desc_lo_kmajor(smem_u32(sdO));
+            const uint32_t k_lo = desc_lo_kmajor(smem_u32(sK)), v_lo = desc_lo_kmajor(smem_u32(sV));
+            const uint32_t kt_lo = desc_lo_mnmajor(smem_u32(sK), kPanel);
             auto issue_s = [&](int e) -> bool {             // S(e) = Q K(e)^T into the ping/pong buffer e & 1
-                const int s = e % C::kStages;
-                if (!mbar_wait(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
+                const int s = e % C::kStagesK;
+                if (!mbar_wait_warp(&bar.a_full[s], (uint32_t)(e / C::kStagesK) & 1u, abortp)) return false;
                 tc_fence_after();
-                const uint32_t ka = k_addr + s * C::kTile;
+                const uint32_t ka = k_lo + s * (C::kTile >> 4);
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k) {
-                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
-                    mma_ss(tmem + kColS + (e & 1) * 128, desc_kmajor(q_addr + off), desc_kmajor(ka + off), C::kIdescS, k > 0);
-                }
-                mma_commit(&bar.s_full[e & 1]);
+                for (int k = 0; k < DH / 16; ++k)
+                    mma_ss_elect(tmem + kColS + (e & 1) * 128, make_desc(q_lo + kstep_off(k, kPanel)), make_desc(ka + kstep_off(k, kPanel)),
+                           C::kIdescS, k > 0);
+                mma_commit_elect(&bar.s_full[e & 1]);
                 return true;
             };
             if (ok) ok = issue_s(0);
             for (int e = 0; e < E && ok; ++e) {
-                const int s = e % C::kStages;
-                if (!mbar_wait(&bar.b_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) { ok = false; break; }
+                const int s = e % C::kStagesK, sv = e % C::kStages;
+                if (!mbar_wait_warp(&bar.b_full[sv], (uint32_t)(e / C::kStages) & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t ka = k_addr + s * C::kTile, va = v_addr + s * C::kTile;
+                const uint32_t va = v_lo + sv * (C::kTile >> 4), kta = kt_lo + s * (C::kTile >> 4);
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k) {        // dP(e) = dO V(e)^T  (dS(e-1), which shares the columns, was consumed by dQ(e-1) issued before)
-                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
-                    mma_ss(tmem + kColDP, desc_kmajor(g_addr + off), desc_kmajor(va + off), C::kIdescS, k > 0);
-                }
-                mma_commit(&bar.dp_full);
-                mma_commit(&bar.b_empty[s]);
+                for (int k = 0; k < DH / 16; ++k)          // dP(e) = dO V(e)^T  (dS(e-1), which shares the columns, was consumed by dQ(e-1) issued before)
+                    mma_ss_elect(tmem + kColDP, make_desc(g_lo + kstep_off(k, kPanel)), make_desc(va + kstep_off(k, kPanel)), C::kIdescS, k > 0);
+                mma_commit_elect(&bar.dp_full);
+                mma_commit_elect(&bar.b_empty[sv]);
                 if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
-                if (!mbar_wait(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                if (!mbar_wait_warp(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < kBlk / 16; ++k)         // dQ += dS(e) K(e)
-                    mma_ts(tmem + kColAcc, tmem + kColDP + packed_half_col(k), desc_mnmajor(ka + k * 2048, kPanel), C::kIdescAcc,
+                    mma_ts_elect(tmem + kColAcc, tmem + kColDP + packed_half_col(k), make_desc(kta + k * (2048 >> 4)), C::kIdescAcc,
                            (e > 0 || k > 0) ? 1u : 0u);
-                mma_commit(&bar.a_empty[s]);
+                mma_commit_elect(&bar.a_empty[s]);
             }
-            if (ok) mma_commit(&bar.acc_done);
+            if (ok) mma_commit_elect(&bar.acc_done);
         }
     } else {
         // ------------------------------------------------------------ element-wise warpgroups (thread = query row, 64 of the 128 columns)
@@ -434,7 +436,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
     const int b = blockIdx.z, h = blockIdx.y;
     const long long bh = (long long)b * p.H + h;
     // key tiles in decreasing order of work: L3 (seen by every query), L2 from the oldest key on, L1
@@ -505,54 +508,53 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                 mbar_wait(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
     } else if (warp == kMmaWarp) {
-        if (lane == 0 && E > 0) {
-            bool ok = mbar_wait(&bar.fixed_full, 0, abortp);
+        if (E > 0) {   // every lane runs the issue loop (converged); elect.sync inside the wrappers picks the issuing lane
+            bool ok = mbar_wait_warp(&bar.fixed_full, 0, abortp);
             tc_fence_after();
-            const uint32_t k_addr = smem_u32(sK), v_addr = smem_u32(sV), q_addr = smem_u32(sQ), g_addr = smem_u32(sdO);
+            // low descriptor words (see make_desc): K-major views for S^T and dP^T, MN-major views of Q and dO for dK and dV
+            const uint32_t k_lo = desc_lo_kmajor(smem_u32(sK)), v_lo = desc_lo_kmajor(smem_u32(sV));
+            const uint32_t q_lo = desc_lo_kmajor(smem_u32(sQ)), g_lo = desc_lo_kmajor(smem_u32(sdO));
+            const uint32_t qt_lo = desc_lo_mnmajor(smem_u32(sQ), kPanel), gt_lo = desc_lo_mnmajor(smem_u32(sdO), kPanel);
             auto issue_s = [&](int e) -> bool {             // S^T(e) = K Q(e)^T   (P^T(e-1), which shares the columns, was consumed by dV(e-1) issued before)
                 const int s = e % C::kStages;
-                if (!mbar_wait(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
+                if (!mbar_wait_warp(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
                 tc_fence_after();
-                const uint32_t qa = q_addr + s * C::kTile;
+                const uint32_t qa = q_lo + s * (C::kTile >> 4);
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k) {
-                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
-                    mma_ss(tmem + kColS, desc_kmajor(k_addr + off), desc_kmajor(qa + off), C::kIdescS, k > 0);
-                }
-                mma_commit(&bar.s_full[0]);
+                for (int k = 0; k < DH / 16; ++k)
+                    mma_ss_elect(tmem + kColS, make_desc(k_lo + kstep_off(k, kPanel)), make_desc(qa + kstep_off(k, kPanel)), C::kIdescS, k > 0);
+                mma_commit_elect(&bar.s_full[0]);
                 return true;
             };
             auto issue_dp = [&](int e) {                    // dP^T(e) = V dO(e)^T  (its stage was awaited by issue_s(e))
-                const uint32_t ga = g_addr + (e % C::kStages) * C::kTile;
+                const uint32_t ga = g_lo + (e % C::kStages) * (C::kTile >> 4);
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k) {
-                    const uint32_t off = (k / 4) * kPanel + (k % 4) * 32;
-                    mma_ss(tmem + kColDP, desc_kmajor(v_addr + off), desc_kmajor(ga + off), C::kIdescS, k > 0);
-                }
-                mma_commit(&bar.dp_full);
+                for (int k = 0; k < DH / 16; ++k)
+                    mma_ss_elect(tmem + kColDP, make_desc(v_lo + kstep_off(k, kPanel)), make_desc(ga + kstep_off(k, kPanel)), C::kIdescS, k > 0);
+                mma_commit_elect(&bar.dp_full);
             };
             if (ok) ok = issue_s(0);
             if (ok) issue_dp(0);
             for (int e = 0; e < E && ok; ++e) {
                 const int s = e % C::kStages;
-                const uint32_t qa = q_addr + s * C::kTile, ga = g_addr + s * C::kTile;
-                if (!mbar_wait(&bar.p_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                const uint32_t qta = qt_lo + s * (C::kTile >> 4), gta = gt_lo + s * (C::kTile >> 4);
+                if (!mbar_wait_warp(&bar.p_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < kBlk / 16; ++k)         // dV += P^T(e) dO(e)
-                    mma_ts(tmem + kColDV, tmem + kColS + packed_half_col(k), desc_mnmajor(ga + k * 2048, kPanel), C::kIdescAcc,
+                    mma_ts_elect(tmem + kColDV, tmem + kColS + packed_half_col(k), make_desc(gta + k * (2048 >> 4)), C::kIdescAcc,
                            (e > 0 || k > 0) ? 1u : 0u);
                 if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
-                if (!mbar_wait(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                if (!mbar_wait_warp(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < kBlk / 16; ++k)         // dK += dS^T(e) Q(e)
-                    mma_ts(tmem + kColDK, tmem + kColDP + packed_half_col(k), desc_mnmajor(qa + k * 2048, kPanel), C::kIdescAcc,
+                    mma_ts_elect(tmem + kColDK, tmem + kColDP + packed_half_col(k), make_desc(qta + k * (2048 >> 4)), C::kIdescAcc,
                            (e > 0 || k > 0) ? 1u : 0u);
-                mma_commit(&bar.a_empty[s]);
+                mma_commit_elect(&bar.a_empty[s]);
                 if (e + 1 < E) issue_dp(e + 1);
             }
-            if (ok) mma_commit(&bar.acc_done);
+            if (ok) mma_commit_elect(&bar.acc_done);
         }
     } else {
         // ------------------------------------------------------------ element-wise warpgroups (thread = key row, 64 of the 128 query columns)

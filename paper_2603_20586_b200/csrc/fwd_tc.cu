@@ -14,7 +14,7 @@
 //                    running maximum grows by more than 2^8 (lazy rescale), and does the epilogue.
 //   warp 8           producer: one lane issues the TMA loads of Q and of the K / V tile list into
 //                    128-byte-swizzled shared-memory rings (one mbarrier pair per stage).
-//   warp 9           one lane issues every tcgen05.mma: S_q = Q_q K^T (both operands from shared
+//   warp 9           issues every tcgen05.mma (the warp runs its loop converged, one elected lane issues): S_q = Q_q K^T (both operands from shared
 //                    memory) and O_q += P_q V (P from TMEM, V from shared memory, N-major), in the
 //                    order  S0(e)  O1(e-1)  S1(e)  O0(e)  so that each warpgroup's softmax overlaps
 //                    the other tile's matrix products.
@@ -89,7 +89,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
     const int b = blockIdx.z, h = blockIdx.y;
     const int qpair = gridDim.x - 1 - blockIdx.x;          // heaviest (latest) rows first
     const long long m0 = (long long)qpair * (kNumQ * kTileM);
@@ -164,53 +165,54 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 mbar_wait(&bar.v_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
     } else if (warp == kMmaWarp) {
-        if (lane == 0) {
-            bool ok = mbar_wait(&bar.q_full, 0, abortp);
+        {   // every lane runs the issue loop (converged); elect.sync inside the wrappers picks the issuing lane
+            bool ok = mbar_wait_warp(&bar.q_full, 0, abortp);
             tc_fence_after();
-            const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+            // low descriptor words of the operands (see make_desc)
+            const uint32_t q_lo = desc_lo_kmajor(smem_u32(sQ)), k_lo = desc_lo_kmajor(smem_u32(sK));
+            const uint32_t v_lo = desc_lo_mnmajor(smem_u32(sV), kPanelBytes);
             auto issue_qk = [&](int q, int s) {
-                const uint32_t qa = q_addr + q * C::kTileBytes, ka = k_addr + s * C::kTileBytes;
+                const uint32_t qa = q_lo + q * (C::kTileBytes >> 4), ka = k_lo + s * (C::kTileBytes >> 4);
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k) {
-                    const uint32_t off = (k / 4) * kPanelBytes + (k % 4) * 32;
-                    mma_ss(tmem + q * kTileN, desc_kmajor(qa + off), desc_kmajor(ka + off), C::kIdescQK, k > 0);
-                }
-                mma_commit(&bar.s_full[q]);
+                for (int k = 0; k < DH / 16; ++k)
+                    mma_ss_elect(tmem + q * kTileN, make_desc(qa + kstep_off(k, kPanelBytes)), make_desc(ka + kstep_off(k, kPanelBytes)),
+                           C::kIdescQK, k > 0);
+                mma_commit_elect(&bar.s_full[q]);
             };
             auto issue_pv = [&](int q, int s, bool accumulate) {
-                const uint32_t va = v_addr + s * C::kTileBytes;
+                const uint32_t va = v_lo + s * (C::kTileBytes >> 4);
 #pragma unroll
                 for (int k = 0; k < kTileN / 16; ++k)
-                    mma_ts(tmem + 256 + q * DH, tmem + q * kTileN + k * 8, desc_mnmajor(va + k * 2048, kPanelBytes), C::kIdescPV,
+                    mma_ts_elect(tmem + 256 + q * DH, tmem + q * kTileN + k * 8, make_desc(va + k * (2048 >> 4)), C::kIdescPV,
                            (accumulate || k > 0) ? 1u : 0u);
-                mma_commit(&bar.pv_done[q]);
+                mma_commit_elect(&bar.pv_done[q]);
             };
             for (int e = 0; e < E && ok; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
-                if (!mbar_wait(&bar.k_full[s], ph, abortp)) { ok = false; break; }
+                if (!mbar_wait_warp(&bar.k_full[s], ph, abortp)) { ok = false; break; }
                 tc_fence_after();
                 issue_qk(0, s);
                 if (e > 0) {
                     const int sp = (e - 1) % C::kStages;
-                    if (!mbar_wait(&bar.p_full[1], (uint32_t)(e - 1) & 1u, abortp)) { ok = false; break; }
+                    if (!mbar_wait_warp(&bar.p_full[1], (uint32_t)(e - 1) & 1u, abortp)) { ok = false; break; }
                     tc_fence_after();
                     issue_pv(1, sp, e - 1 > 0);
-                    mma_commit(&bar.v_empty[sp]);
+                    mma_commit_elect(&bar.v_empty[sp]);
                 }
                 issue_qk(1, s);
-                mma_commit(&bar.k_empty[s]);
-                if (!mbar_wait(&bar.v_full[s], ph, abortp)) { ok = false; break; }
-                if (!mbar_wait(&bar.p_full[0], (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                mma_commit_elect(&bar.k_empty[s]);
+                if (!mbar_wait_warp(&bar.v_full[s], ph, abortp)) { ok = false; break; }
+                if (!mbar_wait_warp(&bar.p_full[0], (uint32_t)e & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
                 issue_pv(0, s, e > 0);
             }
             if (ok && E > 0) {
                 const int sp = (E - 1) % C::kStages;
-                if (mbar_wait(&bar.p_full[1], (uint32_t)(E - 1) & 1u, abortp)) {
+                if (mbar_wait_warp(&bar.p_full[1], (uint32_t)(E - 1) & 1u, abortp)) {
                     tc_fence_after();
                     issue_pv(1, sp, E - 1 > 0);
-                    mma_commit(&bar.v_empty[sp]);
+                    mma_commit_elect(&bar.v_empty[sp]);
                 }
             }
         }

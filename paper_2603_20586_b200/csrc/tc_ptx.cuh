@@ -67,6 +67,45 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, 
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// The same descriptors split into their two 32-bit words.  The high word is one constant for every operand of
+// these kernels; the low word is the start-address field (address >> 4: shared-memory addresses are
+// below 256 KB, so the 14-bit field cannot overflow and byte offsets are simply added as offset >> 4)
+// plus the leading-dimension field.  The issuing warp then spends one add per operand and matrix product.
+constexpr uint32_t kDescHi = 64u | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo_kmajor(uint32_t addr) { return (addr >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mnmajor(uint32_t addr, uint32_t panel_stride_bytes) {
+    return (addr >> 4) | ((panel_stride_bytes >> 4) << 16);
+}
+__device__ __forceinline__ uint64_t make_desc(uint32_t lo) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(kDescHi));
+    return d;
+}
+// offset (in descriptor units of 16 bytes) of K-step k inside a K-major tile whose 64-column panels are `panel` bytes apart
+__device__ __forceinline__ constexpr uint32_t kstep_off(int k, uint32_t panel) {
+    return ((uint32_t)(k / 4) * panel + (uint32_t)(k % 4) * 32u) >> 4;
+}
+// The matrix-product and commit instructions for a warp that runs its issue loop CONVERGED: every lane executes
+// the block and elect.sync picks the one lane that issues.  Kept converged, the compiler can hold descriptors
+// and addresses in uniform registers; issued from inside an `if (lane == 0)` region every operand has to be
+// moved there first, which was measured at about 70 cycles per instruction -- more than the 64 cycles a
+// 128x128x16 product takes to execute -- against at most 34 cycles this way.
+__device__ __forceinline__ void mma_ss_elect(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p, q;\nelect.sync _|q, 0xffffffff;\nsetp.ne.b32 p, %4, 0;\n@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_ts_elect(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p, q;\nelect.sync _|q, 0xffffffff;\nsetp.ne.b32 p, %4, 0;\n@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit_elect(uint64_t* bar) {
+    asm volatile("{\n.reg .pred q;\nelect.sync _|q, 0xffffffff;\n@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}"
+                 ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait executed by every lane of a converged warp; the result is made warp-uniform.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag));
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
