@@ -45,7 +45,8 @@ struct BwdMaps {
 
 struct BwdTcParams {
     __nv_bfloat16* dQ;
-    const float2* stats[3];   // per level: [B*H, Tpad] of {D_t, log2(lambda_{t,l}) - LSE_t log2(e)}
+    const float* statD;       // [B*H, Tpad]  D_t = dO_t . O_t
+    const float* statB[3];    // per level: [B*H, Tpad]  log2(lambda_{t,l}) - LSE_t log2(e)  (-inf on padding rows)
     float* Gpart;             // [B, H, T, 3]
     LevelGradDev dL[3];
     long long n[3];
@@ -61,7 +62,7 @@ struct BCfg {
     static constexpr int kPanels = DH / 64;
     static constexpr uint32_t kTile = kPanels * kPanel;       // a 128-row tile
     static constexpr int kStages = DH == 128 ? 2 : 4;         // also keeps the CTA above half of shared memory
-    static constexpr uint32_t kStatBytes = kBlk * sizeof(float2);
+    static constexpr uint32_t kStatBytes = 2 * kBlk * sizeof(float);   // per stage: D and the level's bias of 128 queries
     static constexpr int kStagesK = DH == 128 ? 3 : 4;        // K ring of the dQ kernel: K(e) stays in use until dQ(e), two tiles after it is first read
     static constexpr uint32_t kSmemDq = 2 * kTile + (kStages + kStagesK) * kTile + 1024;
     static constexpr uint32_t kSmemDkv = 2 * kTile + kStages * (2 * kTile + kStatBytes) + 1024;
@@ -93,14 +94,14 @@ __device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1,
 template <int DH>
 __global__ void __launch_bounds__(256) bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
                                                        const float* __restrict__ LSE, const float* __restrict__ gate, int H,
-                                                       int T, int Tpad, long long rows_pad, float2* __restrict__ s0,
-                                                       float2* __restrict__ s1, float2* __restrict__ s2) {
+                                                       int T, int Tpad, long long rows_pad, float* __restrict__ sD,
+                                                       float* __restrict__ b0, float* __restrict__ b1, float* __restrict__ b2) {
     const int lane = threadIdx.x & 31;
     const long long r = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (r >= rows_pad) return;
     const long long bh = r / Tpad;
     const int t = (int)(r % Tpad);
-    float2 o0 = make_float2(0.f, -INFINITY), o1 = o0, o2 = o0;
+    float dsum = 0.f, o0 = -INFINITY, o1 = -INFINITY, o2 = -INFINITY;
     if (t < T) {
         const long long row = bh * T + t;
         constexpr int PER = DH / 32;                   // 2 or 4 consecutive elements per lane
@@ -119,11 +120,12 @@ __global__ void __launch_bounds__(256) bwd_prep_kernel(const __nv_bfloat16* __re
         const float* g = gate + ((bh / H) * T + t) * 3;
         const bool live = lse > -INFINITY;
         const float l2 = lse * kLog2e;
-        o0 = make_float2(s, (live && g[0] > 0.f) ? log2f(g[0]) - l2 : -INFINITY);
-        o1 = make_float2(s, (live && g[1] > 0.f) ? log2f(g[1]) - l2 : -INFINITY);
-        o2 = make_float2(s, (live && g[2] > 0.f) ? log2f(g[2]) - l2 : -INFINITY);
+        dsum = s;
+        o0 = (live && g[0] > 0.f) ? log2f(g[0]) - l2 : -INFINITY;
+        o1 = (live && g[1] > 0.f) ? log2f(g[1]) - l2 : -INFINITY;
+        o2 = (live && g[2] > 0.f) ? log2f(g[2]) - l2 : -INFINITY;
     }
-    if (lane == 0) { s0[r] = o0; s1[r] = o1; s2[r] = o2; }
+    if (lane == 0) { sD[r] = dsum; b0[r] = o0; b1[r] = o1; b2[r] = o2; }
 }
 
 // Key tile range [first, end) (128-row units) of query rows [r0, r1] on one level.
@@ -295,11 +297,10 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
         const uint32_t dp_addr = tmem + lane_base + kColDP + w * 64;
         float Dt = 0.f, bias[3] = {-INFINITY, -INFINITY, -INFINITY};
         if (row_valid) {
+            Dt = p.statD[bh * p.Tpad + t];
 #pragma unroll
             for (int l = 0; l < 3; ++l) {
-                const float2 sv = p.stats[l][bh * p.Tpad + t];
-                Dt = sv.x;
-                bias[l] = sv.y;
+                bias[l] = p.statB[l][bh * p.Tpad + t];
             }
         }
         float Al[3] = {0.f, 0.f, 0.f}, Sl[3] = {0.f, 0.f, 0.f};   // per level: sum p dP and sum p over this thread's columns
@@ -431,7 +432,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     uint8_t* sV = sK + C::kTile;
     uint8_t* sQ = sV + C::kTile;                          // kStages tiles
     uint8_t* sdO = sQ + C::kStages * C::kTile;            // kStages tiles
-    float2* sStat = reinterpret_cast<float2*>(sdO + C::kStages * C::kTile);   // kStages x 128
+    float* sStat = reinterpret_cast<float*>(sdO + C::kStages * C::kTile);     // kStages x {D[128], bias[128]}
     __shared__ BwdBarriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -488,7 +489,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                 tma_load_4d(sK + pn * kPanel, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
                 tma_load_4d(sV + pn * kPanel, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
             }
-            const float2* stat = p.stats[lvl] + bh * p.Tpad;
+            const float* statD = p.statD + bh * p.Tpad;
+            const float* statB = p.statB[lvl] + bh * p.Tpad;
             for (int e = 0; e < E; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
@@ -500,7 +502,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                     tma_load_4d(sQ + s * C::kTile + pn * kPanel, &maps.q, pn * 64, tt, h, b, &bar.a_full[s]);
                     tma_load_4d(sdO + s * C::kTile + pn * kPanel, &maps.dO, pn * 64, tt, h, b, &bar.a_full[s]);
                 }
-                bulk_load(sStat + s * kBlk, stat + tt, C::kStatBytes, &bar.a_full[s]);
+                bulk_load(sStat + s * 2 * kBlk, statD + tt, kBlk * sizeof(float), &bar.a_full[s]);
+                bulk_load(sStat + s * 2 * kBlk + kBlk, statB + tt, kBlk * sizeof(float), &bar.a_full[s]);
                 ++issued;
             }
             mbar_wait(&bar.fixed_full, 0, abortp);
@@ -576,7 +579,20 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
         for (int e = 0; e < E; ++e) {
             const int s = e % C::kStages;
             const long long tt = (long long)(first + e) * kBlk;        // first query of the tile
-            const float4* stat = reinterpret_cast<const float4*>(sStat + s * kBlk + w * 64);   // {D, bias} of two queries per load
+            // The per-query statistics of the tile sit in this stage's shared memory; fetch this thread's 64 biases
+            // before waiting for S so that the loads' latency (long while the tensor pipe saturates shared
+            // memory) is off the path.  The stage's own barrier has long completed; waiting on it orders the reads.
+            ok = mbar_wait(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const float4* statD4 = reinterpret_cast<const float4*>(sStat + s * 2 * kBlk + w * 64);
+            const float4* statB4 = reinterpret_cast<const float4*>(sStat + s * 2 * kBlk + kBlk + w * 64);
+            float st[64];
+#pragma unroll
+            for (int c = 0; c < 64; c += 4) {
+                const float4 v4 = statB4[c / 4];
+                st[c] = v4.x; st[c + 1] = v4.y; st[c + 2] = v4.z; st[c + 3] = v4.w;
+            }
             // phase 1: P^T = 2^(s * scale + bias_t) for this thread's 64 query columns
             ok = mbar_wait(&bar.s_full[0], (uint32_t)e & 1u, abortp);
             ok = __all_sync(0xffffffffu, ok);
@@ -598,15 +614,17 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                 for (int c = 0; c < 64; ++c)
                     if (c < c_lo || c >= c_hi) pr[c] = -INFINITY;
             }
-            uint32_t pk[32];
+            uint32_t pk[32];        // P^T rounded to bf16; phase 2 uses these same rounded values
 #pragma unroll
-            for (int c = 0; c < 64; c += 2) {
-                const float4 sv = stat[c / 2];
-                pr[c] = ex2(fmaf(pr[c], p.scale_log2, sv.y));
-                pr[c + 1] = ex2(fmaf(pr[c + 1], p.scale_log2, sv.w));
-                pk[c / 2] = pack_bf16(pr[c], pr[c + 1]);
-            }
+            for (int c = 0; c < 64; c += 2)
+                pk[c / 2] = pack_bf16(ex2(fmaf(pr[c], p.scale_log2, st[c])), ex2(fmaf(pr[c + 1], p.scale_log2, st[c + 1])));
             tmem_st32(s_addr, pk);
+            // D_t of the 64 queries, again ahead of the wait
+#pragma unroll
+            for (int c = 0; c < 64; c += 4) {
+                const float4 v4 = statD4[c / 4];
+                st[c] = v4.x; st[c + 1] = v4.y; st[c + 2] = v4.z; st[c + 3] = v4.w;
+            }
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(&bar.p_full);
@@ -615,14 +633,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            float dp[64];
-            tmem_ld32(dp_addr, reinterpret_cast<uint32_t*>(dp));
-            tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(dp) + 32);
+            tmem_ld32(dp_addr, reinterpret_cast<uint32_t*>(pr));
+            tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(pr) + 32);
             tmem_ld_wait();
 #pragma unroll
             for (int c = 0; c < 64; c += 2) {
-                const float4 sv = stat[c / 2];
-                pk[c / 2] = pack_bf16(pr[c] * (dp[c] - sv.x), pr[c + 1] * (dp[c + 1] - sv.z));
+                const float p0 = __uint_as_float(pk[c / 2] << 16), p1 = __uint_as_float(pk[c / 2] & 0xffff0000u);
+                pk[c / 2] = pack_bf16(p0 * (pr[c] - st[c]), p1 * (pr[c + 1] - st[c + 1]));
             }
             tmem_st32(dp_addr, pk);
             tmem_st_wait();
@@ -665,21 +682,23 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
     using C = BCfg<DH>;
     const int Tpad = (bp.T + kBlk - 1) / kBlk * kBlk;
     const long long rows_pad = (long long)bp.B * bp.H * Tpad;
-    float2* stats[3];
-    for (int l = 0; l < 3; ++l) stats[l] = reinterpret_cast<float2*>(bp.stats) + (long long)l * rows_pad;
+    float* statD = bp.stats;                              // the workspace holds D and the three bias arrays back to back
+    float* statB[3];
+    for (int l = 0; l < 3; ++l) statB[l] = bp.stats + (long long)(1 + l) * rows_pad;
     const long long sq_n = DH, sq_h = (long long)bp.T * DH, sq_b = (long long)bp.H * bp.T * DH;
 
     bwd_prep_kernel<DH><<<(unsigned)((rows_pad + 7) / 8), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(bp.O), static_cast<const __nv_bfloat16*>(bp.dO), bp.LSE, bp.gate, bp.H, bp.T, Tpad,
-        rows_pad, stats[0], stats[1], stats[2]);
+        rows_pad, statD, statB[0], statB[1], statB[2]);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
     BwdTcParams p;
     p.dQ = static_cast<__nv_bfloat16*>(bp.dQ);
+    p.statD = statD;
     p.Gpart = bp.Gpart;
     for (int l = 0; l < 3; ++l) {
-        p.stats[l] = stats[l];
+        p.statB[l] = statB[l];
         p.dL[l] = bp.dL[l];
         p.n[l] = bp.L[l].n;
         p.kv_tiles[l] = (int)((bp.L[l].n + 127) / 128);

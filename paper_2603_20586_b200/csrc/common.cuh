@@ -110,7 +110,7 @@ struct BwdParams {
     float* dG;        // [B,T,3]
     float* delta;     // ws: [B,H,T]
     float* Gpart;     // ws: [B,H,T,3]
-    float* stats;     // ws: 3 x [B,H,Tpad] float2 (tensor-core path; Tpad = T rounded up to 128)
+    float* stats;     // ws: room for 6 x [B,H,Tpad] floats (tensor-core path uses 4; Tpad = T rounded up to 128)
     int B, H, T, d;
     int window, q_offset;
     float scale;
