@@ -138,7 +138,7 @@ CONFIGS: Dict[str, WorkloadConfig] = {
     # profiler-sized variants (same per-head geometry, fewer heads / sequences) for ncu captures
     "c3p": WorkloadConfig("c3p", 2, "bf16", 1, 8, 128, 4096, 32768, 4096, (32768, 32768, 8192)),
     "c4p": WorkloadConfig("c4p", 3, "bf16", 2, 32, 128, 4096, 1, 4096, (4096, 32768, 8192), decode=True),
-    "c5p": WorkloadConfig("c5p", 4, "bf16", 1, 4, 128, 2048, 8192, 1024, (8192, 8192, 2048)),
+    "c5p": WorkloadConfig("c5p", 4, "bf16", 1, 16, 128, 2048, 8192, 1024, (8192, 8192, 2048)),
 }
 
 
