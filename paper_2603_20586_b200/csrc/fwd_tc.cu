@@ -18,7 +18,9 @@
 //                    memory) and O_q += P_q V (P from TMEM, V from shared memory, N-major), in the
 //                    order  S0(e)  O1(e-1)  S1(e)  O0(e)  so that each warpgroup's softmax overlaps
 //                    the other tile's matrix products.
-// TMEM: columns [0,128) S0/P0, [128,256) S1/P1, [256,256+d) O0, [256+d,256+2d) O1.
+// TMEM: columns [0,128) S0/P0, [128,256) S1/P1, [256,256+d) O0, [256+d,256+2d) O1.  With d = 64 the 128 columns
+// left over hold P0 and P1 on their own ([384,448), [448,512)), and S_q(e+1) is multiplied while the softmax of
+// S_q(e) runs (the hand-off is "S is in registers", not "P has been consumed").
 // Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA raises a flag in shared
 // memory, writes the device status word, lets every role drain, frees TMEM and returns.
 #include "tc_ptx.cuh"
@@ -56,6 +58,10 @@ struct Cfg {
     static constexpr int kStages = DH == 128 ? 2 : 4;
     static constexpr uint32_t kSmemBytes = (kNumQ + 2 * kStages) * kTileBytes + 1024;
     static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    // With d = 64 the two O accumulators leave 128 TMEM columns free: P gets a region of its own there instead of
+    // overwriting S, so S(e+1) can be multiplied while the softmax of S(e) is still running.
+    static constexpr bool kSeparateP = DH == 64;
+    static constexpr uint32_t kColP = 256 + kNumQ * DH;       // first P column when kSeparateP
     static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 };
 
@@ -63,6 +69,7 @@ struct Barriers {
     uint64_t q_full;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
     uint64_t s_full[kNumQ], p_full[kNumQ], pv_done[kNumQ];
+    uint64_t s_free[kNumQ];   // d = 64 only: the warpgroup has read S(e) into registers, S(e+1) may overwrite it
 };
 
 // Key-tile range [first, end) of a block of query rows [r0, r1] (inclusive) on one level.
@@ -105,6 +112,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         }
         for (int q = 0; q < kNumQ; ++q) {
             mbar_init(&bar.s_full[q], 1); mbar_init(&bar.p_full[q], kTileM); mbar_init(&bar.pv_done[q], 1);
+            mbar_init(&bar.s_free[q], kTileM);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -183,10 +191,43 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 const uint32_t va = v_lo + s * (C::kTileBytes >> 4);
 #pragma unroll
                 for (int k = 0; k < kTileN / 16; ++k)
-                    mma_ts_elect(tmem + 256 + q * DH, tmem + q * kTileN + k * 8, make_desc(va + k * (2048 >> 4)), C::kIdescPV,
-                           (accumulate || k > 0) ? 1u : 0u);
+                    mma_ts_elect(tmem + 256 + q * DH, tmem + (C::kSeparateP ? C::kColP + q * (kTileN / 2) : q * kTileN) + k * 8,
+                                 make_desc(va + k * (2048 >> 4)), C::kIdescPV, (accumulate || k > 0) ? 1u : 0u);
                 mma_commit_elect(&bar.pv_done[q]);
             };
+            if (C::kSeparateP) {
+                // S_q(e+1) is issued as soon as the warpgroup has S_q(e) in registers; O_q += P_q(e) V(e) when P_q(e) is written.
+                if (ok && E > 0) ok = mbar_wait_warp(&bar.k_full[0], 0, abortp);
+                if (ok && E > 0) {
+                    tc_fence_after();
+                    issue_qk(0, 0);
+                    issue_qk(1, 0);
+                    mma_commit_elect(&bar.k_empty[0]);
+                }
+                for (int e = 0; e < E && ok; ++e) {
+                    const int s = e % C::kStages, sn = (e + 1) % C::kStages;
+                    if (e + 1 < E) {
+                        if (!mbar_wait_warp(&bar.k_full[sn], (uint32_t)((e + 1) / C::kStages) & 1u, abortp)) { ok = false; break; }
+#pragma unroll
+                        for (int q = 0; q < kNumQ; ++q) {
+                            if (!mbar_wait_warp(&bar.s_free[q], (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                            tc_fence_after();
+                            issue_qk(q, sn);
+                        }
+                        if (!ok) break;
+                        mma_commit_elect(&bar.k_empty[sn]);
+                    }
+                    if (!mbar_wait_warp(&bar.v_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) { ok = false; break; }
+#pragma unroll
+                    for (int q = 0; q < kNumQ; ++q) {
+                        if (!mbar_wait_warp(&bar.p_full[q], (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                        tc_fence_after();
+                        issue_pv(q, s, e > 0);
+                    }
+                    if (!ok) break;
+                    mma_commit_elect(&bar.v_empty[s]);
+                }
+            } else {
             for (int e = 0; e < E && ok; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
@@ -215,6 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     mma_commit_elect(&bar.v_empty[sp]);
                 }
             }
+            }   // !kSeparateP
         }
     } else {
         // ------------------------------------------------------------ softmax warpgroups
@@ -225,6 +267,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t s_addr = tmem + lane_base + q * kTileN;
         const uint32_t o_addr = tmem + lane_base + 256 + q * DH;
+        const uint32_t p_addr = C::kSeparateP ? tmem + lane_base + C::kColP + q * (kTileN / 2) : s_addr;   // where P (bf16) goes
         const long long tq0 = m0 + (long long)q * kTileM;                      // first row of this query tile
         const long long tq1 = (tq0 + kTileM - 1 < p.T - 1) ? tq0 + kTileM - 1 : p.T - 1;
 
@@ -259,6 +302,10 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
 #pragma unroll
                 for (int c0 = 0; c0 < kTileN; c0 += 32) tmem_ld32(s_addr + c0, reinterpret_cast<uint32_t*>(s) + c0);
                 tmem_ld_wait();
+                if (C::kSeparateP) {                         // S(e) is in registers: its TMEM columns may be reused
+                    tc_fence_before();
+                    mbar_arrive(&bar.s_free[q]);
+                }
                 const bool need_mask = !(kt >= full_first && kt < full_end);
                 if (need_mask) {
                     const int c_lo = (int)max(-1LL, min(lo - (long long)kt * kTileN, (long long)kTileN));
@@ -288,8 +335,14 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 }
                 l_run = fmaf(l_run, alpha, sum);
                 m_run = m_use;
-                tmem_st32(s_addr, pk);
-                tmem_st32(s_addr + 32, pk + 32);
+                if (C::kSeparateP && e > 0) {                // P(e-1) must have been consumed before P(e) replaces it
+                    ok = mbar_wait(&bar.pv_done[q], (uint32_t)(e - 1) & 1u, abortp);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                tmem_st32(p_addr, pk);
+                tmem_st32(p_addr + 32, pk + 32);
                 // O accumulator rescale (only when some row of this warp moved its reference maximum)
                 if (e > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                     ok = mbar_wait(&bar.pv_done[q], (uint32_t)(e - 1) & 1u, abortp);
