@@ -232,3 +232,27 @@ def router_bwd(R, dG):
     D = R.shape[-1]
     dW = R.reshape(-1, D).T @ dG.reshape(-1, 3)
     return dW, dG.reshape(-1, 3).sum(0)
+
+
+def route_fuse(levels: Sequence, gate) -> np.ndarray:
+    """Route-fusion of Alg. 2 step 6: X_fused[b, j, :] = sum_l lambda[b, j, l] * L_l[b, j, :], in fp64.
+
+    `levels` holds the three token-aligned level tensors; each is [B, n, D] (the paper's L_1, L_2, L_3) or
+    [B, H, n, d] (their per-head key or value projections: because the projection of Alg. 2 step 7 is linear,
+    fusing the projected levels equals projecting the fused representation), or None for an absent level,
+    which contributes nothing.  `gate` is [B, n, 3]: the gate of the token the row belongs to.
+    Plain definition, three explicit terms; no blocking.
+    """
+    g = _f64(gate)
+    out = None
+    for l in range(3):
+        if levels[l] is None:
+            continue
+        x = _f64(levels[l])
+        w = g[:, :, l]
+        w = w[:, None, :, None] if x.ndim == 4 else w[:, :, None]
+        term = w * x
+        out = term if out is None else out + term
+    if out is None:
+        raise ValueError("no level present")
+    return out
