@@ -175,6 +175,24 @@ mka_status mka_bwd(const mka_shape* shape, const void* Q, const mka_level L[3], 
                    void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Route-fusion with cache write (Alg. 2 steps 6-8).  Alg. 2 mixes the three token-aligned level representations of
+ * every token with that token's own gate BEFORE the key/value projection and appends the projected result to ONE
+ * cache; because the projection is linear the same cache rows are obtained by mixing the projected levels:
+ *     dst.dk[b,h,dst_offset + j,:] = sum_l gate[b,j,l] * L[l].k[b,h,j,:]     (and likewise dv from L[l].v)
+ * for j in [0, n).  Attention over that single cache is then mka_fwd / mka_decode with one level.
+ *   B, H, n, d   sizes; d a multiple of 8 (bf16) or 4 (f32), at most 1024; H = 1 and d = D fuses the level
+ *                representations [B, n, D] themselves (step 6 taken literally)
+ *   L[3]         level sources; each L[l].n must be n, or 0 for an absent level (its gate is then ignored);
+ *                a gate that is exactly 0 drops its level's values whatever they are
+ *   gate         [B, n, 3] f32: the gate of the token the row belongs to
+ *   dst          destinations: dk, dv with their strides; dst->n = rows of the destination (capacity);
+ *                rows [dst_offset, dst_offset + n) are written, nothing else is touched
+ * fp32 accumulation, one rounding to the storage type.  16-byte alignment rules as for the other entry points.
+ */
+mka_status mka_fuse_kv(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype, const mka_level L[3],
+                       const float* gate, const mka_level_grad* dst, int64_t dst_offset, void* stream);
+
+/*
  * Decode for callers that cannot provide scratch memory (the paper has no counterpart; this entry
  * point exists for deployment reasons only).  Same computation, arguments and results as mka_decode,
  * but without `ws`: the per-chunk partials are kept in an 8 MiB array that is compiled into the

@@ -24,7 +24,7 @@ TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
-           "mka_bwd_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes"]
+           "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_decode_static", "mka_decode_static_max_bytes"]
 
 
 class MkaError(RuntimeError):
@@ -82,6 +82,7 @@ def _load() -> ctypes.CDLL:
     lib.mka_decode_static_max_bytes.restype = ctypes.c_size_t
     lib.mka_decode_static_max_bytes.argtypes = []
     lib.mka_fwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level)]
+    lib.mka_fuse_kv.argtypes = [i32, i32, i64, i32, i32, ctypes.POINTER(mka_level), vp, ctypes.POINTER(mka_level_grad), i64, vp]
     lib.mka_bwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level), vp]
     for name in EXPORTS:
         if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes"):
@@ -255,6 +256,23 @@ def mka_bwd(shape: mka_shape, Q, K, V, gate, O, LSE, dO, R=None, dQ=None, dK=Non
 
 def mka_fwd_kernel_kind(shape: mka_shape, K, V) -> int:
     return int(lib.mka_fwd_kernel_kind(ctypes.byref(shape), _levels(K, V)))
+
+
+def mka_fuse_kv(K, V, gate, out_k=None, out_v=None, dst_offset=0, stream=None):
+    """Route-fusion with cache write (Alg. 2 steps 6-8): rows [dst_offset, dst_offset+n) of out_k / out_v receive
+    sum_l gate[b,j,l] * K[l][b,h,j,:] (and V likewise).  K, V: three [B,H,n,d] tensors or None; gate [B,n,3] f32."""
+    ref = next(k for k in K if k is not None)
+    B, H, n, d = ref.shape
+    assert gate.is_contiguous() and gate.dtype == torch.float32 and tuple(gate.shape) == (B, n, 3)
+    if out_k is None:
+        out_k = torch.empty((B, H, dst_offset + n, d), dtype=ref.dtype, device=ref.device)
+    if out_v is None:
+        out_v = torch.empty_like(out_k)
+    assert out_k.stride(3) == 1 and out_v.stride() == out_k.stride() and out_k.dtype == ref.dtype
+    dst = mka_level_grad(out_k.data_ptr(), out_v.data_ptr(), out_k.shape[2], out_k.stride(0), out_k.stride(1), out_k.stride(2))
+    _check(lib.mka_fuse_kv(B, H, n, d, _dt(ref), _levels(K, V), _ptr(gate), ctypes.byref(dst), dst_offset, _stream(stream)),
+           "mka_fuse_kv")
+    return out_k, out_v
 
 
 def mka_bwd_kernel_kind(shape: mka_shape, K, V) -> int:

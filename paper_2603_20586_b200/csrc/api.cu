@@ -283,6 +283,40 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     return MKA_OK;
 }
 
+mka_status mka_fuse_kv(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype, const mka_level L[3], const float* gate,
+                       const mka_level_grad* dst, int64_t dst_offset, void* stream) {
+    if (dtype != MKA_BF16 && dtype != MKA_F32) return MKA_ERR_ARG;
+    if (!L || !dst) return MKA_ERR_ARG;
+    if (B < 0 || H < 0 || n < 0 || dst_offset < 0) return MKA_ERR_SHAPE;
+    const int elems = dtype == MKA_BF16 ? 8 : 4;
+    if (d <= 0 || d > 1024 || d % elems) return MKA_ERR_SHAPE;
+    if (dst->n < dst_offset + n) return MKA_ERR_SHAPE;
+    if (B == 0 || H == 0 || n == 0) return MKA_OK;
+    if (!gate || !dst->dk || !dst->dv) return MKA_ERR_ARG;
+    if (dst->stride_n < d || dst->stride_b < 0 || dst->stride_h < 0) return MKA_ERR_SHAPE;
+    if (!aligned16(dst->dk) || !aligned16(dst->dv) || dst->stride_n % elems || dst->stride_b % elems || dst->stride_h % elems)
+        return MKA_ERR_ALIGN;
+    int present = 0;
+    LevelDev lv[3];
+    for (int l = 0; l < 3; ++l) {
+        if (L[l].n != 0 && L[l].n != n) return MKA_ERR_SHAPE;
+        lv[l].k = L[l].k; lv[l].v = L[l].v; lv[l].n = L[l].n;
+        lv[l].sb = L[l].stride_b; lv[l].sh = L[l].stride_h; lv[l].sn = L[l].stride_n;
+        if (L[l].n == 0) continue;
+        ++present;
+        if (!L[l].k || !L[l].v) return MKA_ERR_ARG;
+        if (L[l].stride_n < d || L[l].stride_b < 0 || L[l].stride_h < 0) return MKA_ERR_SHAPE;
+        if (!aligned16(L[l].k) || !aligned16(L[l].v) || L[l].stride_n % elems || L[l].stride_b % elems || L[l].stride_h % elems)
+            return MKA_ERR_ALIGN;
+    }
+    if (!present) return MKA_ERR_ARG;
+    LevelGradDev out;
+    out.dk = dst->dk; out.dv = dst->dv; out.n = dst->n;
+    out.sb = dst->stride_b; out.sh = dst->stride_h; out.sn = dst->stride_n;
+    cudaError_t e = launch_fuse_kv(lv, out, gate, B, H, n, d, dst_offset, dtype, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
 int32_t mka_bwd_kernel_kind(const mka_shape* s, const mka_level L[3], const mka_level_grad dL[3]) {
     if (check_shape(s, false) != MKA_OK || check_levels(s, L) != MKA_OK || s->mode != MKA_MODE_FAST) return -1;
     BwdParams p;

@@ -119,6 +119,8 @@ cudaError_t launch_bwd_simt(const BwdParams& p, int dtype, cudaStream_t st);
 cudaError_t launch_router_bwd(const void* R, int r_dtype, const float* dG, long long rows, int D, float* dW_r,
                               float* db_r, float* partial, int n_row_chunks, cudaStream_t st);
 
+cudaError_t launch_fuse_kv(const LevelDev L[3], const LevelGradDev& out, const float* gate, int B, int H, long long n, int d,
+                           long long dst_offset, int dtype, cudaStream_t st);
 cudaError_t launch_bwd_dgate(const float* Gpart, int B, int H, long long T, float* dG, cudaStream_t st);
 // Tensor-core (TMA + tcgen05) backward; same contract as the forward below.
 cudaError_t launch_bwd_tc(const BwdParams& p, unsigned int* status_word, cudaStream_t st);
