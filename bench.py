@@ -56,6 +56,7 @@ NCU_TRAFFIC = {
     "fwd_tc_kernel@c3": (376.368896e6 + 67.608320e6, 1 * 8),
     "decode_partial_kernel@c4": (1.476439e9 + 6.574e6, 2 * 32),
     "bwd_dq_tc_kernel@c5": (220.280064e6 + 26.611200e6, 1 * 16),
+    "fuse_kv_kernel@f3": (403.135744e6 + 84.349696e6, 1 * 8),
     "bwd_dkv_tc_kernel@c5": (220.329216e6 + 114.653440e6, 1 * 16),
 }
 
@@ -71,7 +72,9 @@ def algorithmic_work(cfg):
     """Flops / bytes the method itself must do (visible pairs only)."""
     pairs = cfg.visible_pairs_per_head() * cfg.B * cfg.H
     return {"pairs": pairs, "fwd_flops": 4.0 * cfg.d * pairs, "bwd_flops": 10.0 * cfg.d * pairs,
-            "decode_bytes": 2.0 * 2.0 * cfg.d * sum(cfg.N) * cfg.B * cfg.H}
+            "decode_bytes": 2.0 * 2.0 * cfg.d * sum(cfg.N) * cfg.B * cfg.H,
+            # route-fusion: K and V of three levels read, one fused K and V written (2 bytes each), plus the gate
+            "fuse_bytes": 2.0 * (3 + 1) * 2.0 * cfg.d * cfg.T * cfg.B * cfg.H + 12.0 * cfg.B * cfg.T}
 
 
 class ClockSampler:
@@ -130,20 +133,26 @@ class Leg:
             cfg = type(cfg)(**{**cfg.__dict__, "seed": cfg.seed + 1000 * seed_shift})
         self.cfg = cfg
         self.work = algorithmic_work(cfg)
-        self.kind = {"c4": "decode", "c5": "train"}.get(name[:2], "prefill")
+        self.kind = {"c4": "decode", "c5": "train", "f3": "fuse"}.get(name[:2], "prefill")
         names = ["X", "W_r", "Q", "K1", "V1", "K2", "V2", "K3", "V3"] + (["dO"] if self.kind == "train" else [])
+        if self.kind == "fuse":
+            names.remove("Q")
         self.t = {n: make_tensor(cfg, n, device) for n in names}
         B, H, T, d, D = cfg.B, cfg.H, cfg.T, cfg.d, cfg.D
         self.K = [self.t["K1"], self.t["K2"], self.t["K3"]]
         self.V = [self.t["V1"], self.t["V2"], self.t["V3"]]
         self.shape = mka.make_shape(B, H, T, d, D, cfg.W, 0)
         self.gate = torch.empty(B, T, 3, device=device)
-        self.O = torch.empty_like(self.t["Q"])
+        self.O = torch.empty_like(self.t["Q"]) if "Q" in self.t else None
         self.LSE = torch.empty(B, H, T, device=device)
         which = {"decode": mka.MKA_WS_DECODE, "train": mka.MKA_WS_BWD}.get(self.kind, mka.MKA_WS_FWD)
         self.ws = mka.alloc_workspace(self.shape, cfg.N, which, device)
         self.launches = 0
-        if self.kind == "decode":
+        if self.kind == "fuse":
+            self.cache_k, self.cache_v = torch.empty_like(self.K[0]), torch.empty_like(self.V[0])
+            self.ws.zero_()                         # no kernel of this leg writes the status word
+            self.launches_per_step = 2              # router, fuse_kv
+        elif self.kind == "decode":
             self.q = self.t["Q"].view(B, H, d)
             self.Od = torch.empty_like(self.q)
             self.gate_d = self.gate.view(B, 3)
@@ -166,7 +175,9 @@ class Leg:
         mka.mka_router(t["X"], t["W_r"], None, gate=self.gate)
         if record:
             e[1].record()
-        if self.kind == "decode":
+        if self.kind == "fuse":
+            mka.mka_fuse_kv(self.K, self.V, self.gate, out_k=self.cache_k, out_v=self.cache_v)
+        elif self.kind == "decode":
             mka.mka_decode(self.shape, self.q, self.K, self.V, self.gate_d, O=self.Od, LSE=self.LSEd, ws=self.ws)
         else:
             mka.mka_fwd(self.shape, t["Q"], self.K, self.V, self.gate, O=self.O, LSE=self.LSE, ws=self.ws)
@@ -181,6 +192,8 @@ class Leg:
             self.ev.append(e)
 
     def result_tensor(self):
+        if self.kind == "fuse":
+            return self.cache_k
         return self.Od if self.kind == "decode" else (self.grads["dQ"] if self.kind == "train" else self.O)
 
     def kernel_ms(self):
@@ -215,7 +228,14 @@ def timed_steps(leg, steps, warmup, dist=None):
 
 def leg_report(leg, ms_per_step, n_gpus, peaks):
     cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
-    if leg.kind == "decode":
+    if leg.kind == "fuse":
+        achieved = w["fuse_bytes"] / (k["main"] * 1e-3) / 1e9
+        roof = {"kernel": "fuse_kv_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
+                "peak_source": peaks["source"], "traffic": ncu_traffic("fuse_kv_kernel@f3", cfg) if leg.name[:2] == "f3" else None}
+        value = n_gpus * w["fuse_bytes"] / (ms_per_step * 1e-3) / 1e9
+        unit, metric = "GB/s", "route_fuse_hbm_gbs"
+    elif leg.kind == "decode":
         achieved = w["decode_bytes"] / (k["main"] * 1e-3) / 1e9
         roof = {"kernel": "decode_partial_kernel+decode_combine_kernel", "bound": "hbm", "achieved": achieved,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
@@ -315,9 +335,28 @@ def oracle_sample(name, budget_rows=None):
         bytes_ = 2.0 * 2.0 * d * sum(cfg.N) * len(heads)
         return {"value": bytes_ / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle", "seconds": dt,
                 "sample": f"{len(heads)} of {cfg.B * cfg.H} (batch, head) pairs, all {sum(cfg.N)} cached rows each"}
+    if name[:2] == "f3":
+        X, Wr = _router_inputs(cfg)
+        t0 = time.perf_counter()
+        gate, _ = orc.router(X, Wr)
+        dt = time.perf_counter() - t0
+        heads = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(4)]
+        for (b, h) in heads:
+            def sl(nm):
+                off = ((b * cfg.H + h) * cfg.T) * d
+                return make_tensor(cfg, nm, flat_start=off, flat_count=cfg.T * d).double().numpy().reshape(1, 1, cfg.T, d)
+            K = [sl(f"K{l + 1}") for l in range(3)]
+            V = [sl(f"V{l + 1}") for l in range(3)]
+            t0 = time.perf_counter()
+            orc.route_fuse(K, gate[b:b + 1])
+            orc.route_fuse(V, gate[b:b + 1])
+            dt += time.perf_counter() - t0
+        bytes_ = 2.0 * 4 * 2.0 * d * cfg.T * len(heads)
+        return {"value": bytes_ / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dt,
+                "sample": f"{len(heads)} of {cfg.B * cfg.H} (batch, head) pairs, all {cfg.T} rows each (numpy, one thread); router on all tokens"}
     # prefill / training: a few heads, a seeded sample of query rows
-    n_heads = 2
-    n_rows = budget_rows or (1024 if name == "c3" else 2048)
+    n_heads = 2 if budget_rows else 8          # the default sample is sized for roughly 10 s of host work
+    n_rows = budget_rows or 2048
     n_rows = min(n_rows, cfg.T)
     heads = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(n_heads)]
     rows = np.sort(rng.choice(cfg.T, size=n_rows, replace=False))
@@ -352,8 +391,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "c3p", "c4p", "c5p"])
-    ap.add_argument("--legs", default="c4,c5,c2", help="other configurations measured after the primary one ('' = none)")
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "c3p", "c4p", "c5p", "f3p"])
+    ap.add_argument("--legs", default="c4,c5,c2,f3", help="other configurations measured after the primary one ('' = none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -363,7 +402,7 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     cfg = CONFIGS[args.workload]
     wk = args.workload[:2]
-    metric_name = "decode_hbm_gbs" if wk == "c4" else ("fwd_bwd_tflops" if wk == "c5" else "prefill_fwd_tflops")
+    metric_name = {"c4": "decode_hbm_gbs", "c5": "fwd_bwd_tflops", "f3": "route_fuse_hbm_gbs"}.get(wk, "prefill_fwd_tflops")
     base = {"metric": f"FastMKA {metric_name} (algorithmic, visible pairs only)", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
             "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
@@ -416,6 +455,8 @@ def main():
         w = leg.work
         if wk == "c4":
             ev = world * w["decode_bytes"] / (e_ms * 1e-3) / 1e9
+        elif wk == "f3":
+            ev = world * w["fuse_bytes"] / (e_ms * 1e-3) / 1e9
         else:
             ev = world * (w["fwd_flops"] + (w["bwd_flops"] if wk == "c5" else 0.0)) / (e_ms * 1e-3) / 1e12
         out["e2e"] = {"value": ev, "unit": rep["unit"], "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}

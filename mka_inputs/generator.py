@@ -135,6 +135,9 @@ CONFIGS: Dict[str, WorkloadConfig] = {
     "c3": WorkloadConfig("c3", 2, "bf16", 1, 32, 128, 4096, 32768, 4096, (32768, 32768, 8192)),
     "c4": WorkloadConfig("c4", 3, "bf16", 32, 32, 128, 4096, 1, 4096, (4096, 32768, 8192), decode=True),
     "c5": WorkloadConfig("c5", 4, "bf16", 4, 16, 128, 2048, 8192, 1024, (8192, 8192, 2048)),
+    # route-fusion / cache write of Alg. 2 (levels token-aligned): c3's geometry with N_3 = T, and a profiler-sized variant
+    "f3": WorkloadConfig("f3", 5, "bf16", 1, 32, 128, 4096, 32768, 4096, (32768, 32768, 32768)),
+    "f3p": WorkloadConfig("f3p", 5, "bf16", 1, 8, 128, 4096, 32768, 4096, (32768, 32768, 32768)),
     # profiler-sized variants (same per-head geometry, fewer heads / sequences) for ncu captures
     "c3p": WorkloadConfig("c3p", 2, "bf16", 1, 8, 128, 4096, 32768, 4096, (32768, 32768, 8192)),
     "c4p": WorkloadConfig("c4p", 3, "bf16", 2, 32, 128, 4096, 1, 4096, (4096, 32768, 8192), decode=True),
