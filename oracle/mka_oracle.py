@@ -256,3 +256,35 @@ def route_fuse(levels: Sequence, gate) -> np.ndarray:
     if out is None:
         raise ValueError("no level present")
     return out
+
+
+SUMMARY_MEAN, SUMMARY_EMA = 0, 1
+
+
+def l2_summary(X, kind: int = SUMMARY_MEAN, beta: float = 0.9, state=None, n_prev: int = 0):
+    """Causal session summary of Alg. 1 (the loop that fills M_2) / Alg. 2 step 3, in fp64: row t summarises X[:, :t+1].
+
+    kind = SUMMARY_MEAN: prefix mean.  With a carried state (the running SUM of the n_prev earlier tokens of the
+           session) M2[t] = (state + sum_{i<=t} x_i) / (n_prev + t + 1).
+    kind = SUMMARY_EMA:  m_t = beta m_{t-1} + (1 - beta) x_t.  The paper does not say how the average starts; here the
+           first token of a session initialises it (m_0 = x_0); with n_prev > 0 the carried state is m_{-1}.
+    X is [B, T, D].  Returns (M2 [B, T, D], new state [B, D]): the state to carry into the session's next chunk.
+    The recurrences are written out token by token.
+    """
+    X = _f64(X)
+    B, T, D = X.shape
+    M = np.empty_like(X)
+    if kind == SUMMARY_MEAN:
+        run = np.zeros((B, D)) if (state is None or n_prev == 0) else _f64(state).copy()
+        for t in range(T):
+            run = run + X[:, t]
+            M[:, t] = run / float(n_prev + t + 1)
+        return M, run
+    if kind == SUMMARY_EMA:
+        have = state is not None and n_prev > 0
+        m = _f64(state).copy() if have else None
+        for t in range(T):
+            m = X[:, t].copy() if m is None else beta * m + (1.0 - beta) * X[:, t]
+            M[:, t] = m
+        return M, (m if m is not None else np.zeros((B, D)))
+    raise ValueError("unknown summary kind")
