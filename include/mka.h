@@ -192,6 +192,27 @@ mka_status mka_bwd(const mka_shape* shape, const void* Q, const mka_level L[3], 
 mka_status mka_fuse_kv(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype, const mka_level L[3],
                        const float* gate, const mka_level_grad* dst, int64_t dst_offset, void* stream);
 
+/* Causal summaries of mka_l2_summary. */
+typedef enum { MKA_SUMMARY_MEAN = 0, MKA_SUMMARY_EMA = 1 } mka_summary;
+
+/*
+ * L2 session summary (Alg. 1, the loop "M_2[t] <- Summary(X[:, 1:t, :])", named there as "prefix mean or EMA";
+ * Alg. 2 step 3): a causal scan along the sequence that produces the L2 level's source.  Row t of M2 summarises
+ * rows 0..t of X and nothing later:
+ *   MKA_SUMMARY_MEAN   M2[b,t,:] = (S + sum_{i<=t} X[b,i,:]) / (n_prev + t + 1)
+ *   MKA_SUMMARY_EMA    m_t = beta m_{t-1} + (1 - beta) X[b,t,:],  M2[b,t,:] = m_t;  a fresh session starts with m_0 = X[b,0,:]
+ *   X, M2   [B, T, D] contiguous, same dtype (bf16 or f32); D a multiple of 8 (bf16) / 4 (f32); 16-byte aligned
+ *   state   [B, D] f32 or NULL.  With n_prev > 0 it is READ as the session's carried state (MEAN: the running sum S of
+ *           the n_prev earlier tokens; EMA: m_{-1}); with n_prev == 0 the session is fresh and it is ignored on entry.
+ *           When not NULL it is WRITTEN with the state to carry into the session's next chunk.
+ *   beta    EMA decay in [0, 1]; ignored for MEAN
+ *   ws      optional scratch of at least 256 bytes whose first word receives the device status (mka_device_status);
+ *           NULL = no status word
+ * fp32 arithmetic, one rounding to the storage type.  Counts are converted to f32 (exact up to 2^24 tokens).
+ */
+mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_t dtype, int32_t kind, float beta,
+                          float* state, int64_t n_prev, void* M2, void* ws, size_t ws_bytes, void* stream);
+
 /*
  * Decode for callers that cannot provide scratch memory (the paper has no counterpart; this entry
  * point exists for deployment reasons only).  Same computation, arguments and results as mka_decode,

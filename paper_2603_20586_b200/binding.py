@@ -19,12 +19,13 @@ MKA_BF16, MKA_F32 = 0, 1
 MKA_MODE_FAST, MKA_MODE_FULL = 0, 1
 MKA_ROUTE_SOFT, MKA_ROUTE_UNIFORM, MKA_ROUTE_TOP1, MKA_ROUTE_TOP2 = 0, 1, 2, 3
 MKA_FLAG_FORCE_SIMT = 1
+MKA_SUMMARY_MEAN, MKA_SUMMARY_EMA = 0, 1
 MKA_WS_FWD, MKA_WS_DECODE, MKA_WS_BWD = 0, 1, 2
 TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
-           "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_decode_static", "mka_decode_static_max_bytes"]
+           "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_decode_static", "mka_decode_static_max_bytes"]
 
 
 class MkaError(RuntimeError):
@@ -83,6 +84,7 @@ def _load() -> ctypes.CDLL:
     lib.mka_decode_static_max_bytes.argtypes = []
     lib.mka_fwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level)]
     lib.mka_fuse_kv.argtypes = [i32, i32, i64, i32, i32, ctypes.POINTER(mka_level), vp, ctypes.POINTER(mka_level_grad), i64, vp]
+    lib.mka_l2_summary.argtypes = [vp, i32, i64, i32, i32, i32, ctypes.c_float, vp, i64, vp, vp, ctypes.c_size_t, vp]
     lib.mka_bwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level), vp]
     for name in EXPORTS:
         if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes"):
@@ -273,6 +275,21 @@ def mka_fuse_kv(K, V, gate, out_k=None, out_v=None, dst_offset=0, stream=None):
     _check(lib.mka_fuse_kv(B, H, n, d, _dt(ref), _levels(K, V), _ptr(gate), ctypes.byref(dst), dst_offset, _stream(stream)),
            "mka_fuse_kv")
     return out_k, out_v
+
+
+def mka_l2_summary(X, kind=MKA_SUMMARY_MEAN, beta=0.9, state=None, n_prev=0, M2=None, ws=None, stream=None):
+    """Causal L2 session summary of X [B, T, D] (prefix mean or EMA); returns M2.  `state` [B, D] f32 carries a
+    session across calls: read when n_prev > 0, written with the new state whenever it is given."""
+    assert X.dim() == 3 and X.is_contiguous()
+    B, T, D = X.shape
+    if M2 is None:
+        M2 = torch.empty_like(X)
+    assert M2.is_contiguous() and M2.dtype == X.dtype
+    if state is not None:
+        assert state.is_contiguous() and state.dtype == torch.float32 and tuple(state.shape) == (B, D)
+    _check(lib.mka_l2_summary(_ptr(X), B, T, D, _dt(X), kind, float(beta), _ptr(state), n_prev, _ptr(M2), _ptr(ws),
+                              0 if ws is None else ws.numel(), _stream(stream)), "mka_l2_summary")
+    return M2
 
 
 def mka_bwd_kernel_kind(shape: mka_shape, K, V) -> int:

@@ -317,6 +317,27 @@ mka_status mka_fuse_kv(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype
     return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
 }
 
+mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_t dtype, int32_t kind, float beta, float* state,
+                          int64_t n_prev, void* M2, void* ws, size_t ws_bytes, void* stream) {
+    if (dtype != MKA_BF16 && dtype != MKA_F32) return MKA_ERR_ARG;
+    if (kind != MKA_SUMMARY_MEAN && kind != MKA_SUMMARY_EMA) return MKA_ERR_ARG;
+    if (B < 0 || T < 0 || D < 0 || n_prev < 0 || B > 65535) return MKA_ERR_SHAPE;
+    if (T > 0x7fffff00LL) return MKA_ERR_SHAPE;
+    if (D % (dtype == MKA_BF16 ? 8 : 4)) return MKA_ERR_SHAPE;
+    if (kind == MKA_SUMMARY_EMA && !(beta >= 0.f && beta <= 1.f)) return MKA_ERR_ARG;
+    if (B == 0 || T == 0 || D == 0) return MKA_OK;
+    if (!X || !M2) return MKA_ERR_ARG;
+    if (n_prev > 0 && !state) return MKA_ERR_ARG;
+    if (!aligned16(X) || !aligned16(M2)) return MKA_ERR_ALIGN;
+    if (ws && ws_bytes < kWsHeader) return MKA_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (ws && cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
+    cudaError_t e = launch_l2_summary(X, M2, state, n_prev > 0 ? 1 : 0, n_prev, B, T, D, dtype, kind, beta,
+                                      static_cast<unsigned int*>(ws), cs);
+    if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
 int32_t mka_bwd_kernel_kind(const mka_shape* s, const mka_level L[3], const mka_level_grad dL[3]) {
     if (check_shape(s, false) != MKA_OK || check_levels(s, L) != MKA_OK || s->mode != MKA_MODE_FAST) return -1;
     BwdParams p;

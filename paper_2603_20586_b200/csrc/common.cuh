@@ -121,6 +121,8 @@ cudaError_t launch_router_bwd(const void* R, int r_dtype, const float* dG, long 
 
 cudaError_t launch_fuse_kv(const LevelDev L[3], const LevelGradDev& out, const float* gate, int B, int H, long long n, int d,
                            long long dst_offset, int dtype, cudaStream_t st);
+cudaError_t launch_l2_summary(const void* X, void* M2, float* state, int use_state, long long n_prev, int B, long long T, int D,
+                              int dtype, int kind, float beta, unsigned int* status, cudaStream_t st);
 cudaError_t launch_bwd_dgate(const float* Gpart, int B, int H, long long T, float* dG, cudaStream_t st);
 // Tensor-core (TMA + tcgen05) backward; same contract as the forward below.
 cudaError_t launch_bwd_tc(const BwdParams& p, unsigned int* status_word, cudaStream_t st);

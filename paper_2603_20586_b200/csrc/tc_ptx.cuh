@@ -48,6 +48,10 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, i
     asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
                  ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)) : "memory");
+}
 // Shared-memory matrix descriptors (128-byte swizzle; 8-row groups 1024 bytes apart).
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
     return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
@@ -142,5 +146,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 bool make_bf16_map(CUtensorMap* map, const void* base, int d, long long rows, int H, int B, long long sn,
                    long long sh, long long sb, int box_rows);
 bool tensor_map_encoder_available();
+bool make_strip_map(CUtensorMap* map, const void* base, bool is_bf16, int D, long long T, int B, int box_cols, int box_rows);
 
 }  // namespace mka
