@@ -56,6 +56,7 @@ NCU_TRAFFIC = {
     "fwd_tc_kernel@c3": (376.368896e6 + 67.608320e6, 1 * 8),
     "decode_partial_kernel@c4": (1.476439e9 + 6.574e6, 2 * 32),
     "bwd_dq_tc_kernel@c5": (220.280064e6 + 26.611200e6, 1 * 16),
+    "l2_summary_kernel@s3": None,
     "fuse_kv_kernel@f3": (403.135744e6 + 84.349696e6, 1 * 8),
     "bwd_dkv_tc_kernel@c5": (220.329216e6 + 114.653440e6, 1 * 16),
 }
@@ -74,6 +75,8 @@ def algorithmic_work(cfg):
     return {"pairs": pairs, "fwd_flops": 4.0 * cfg.d * pairs, "bwd_flops": 10.0 * cfg.d * pairs,
             "decode_bytes": 2.0 * 2.0 * cfg.d * sum(cfg.N) * cfg.B * cfg.H,
             # route-fusion: K and V of three levels read, one fused K and V written (2 bytes each), plus the gate
+            # L2 summary: X read once, M2 written once
+            "summary_bytes": 2.0 * 2.0 * cfg.D * cfg.T * cfg.B,
             "fuse_bytes": 2.0 * (3 + 1) * 2.0 * cfg.d * cfg.T * cfg.B * cfg.H + 12.0 * cfg.B * cfg.T}
 
 
@@ -133,12 +136,22 @@ class Leg:
             cfg = type(cfg)(**{**cfg.__dict__, "seed": cfg.seed + 1000 * seed_shift})
         self.cfg = cfg
         self.work = algorithmic_work(cfg)
-        self.kind = {"c4": "decode", "c5": "train", "f3": "fuse"}.get(name[:2], "prefill")
+        self.kind = {"c4": "decode", "c5": "train", "f3": "fuse", "s3": "summary"}.get(name[:2], "prefill")
         names = ["X", "W_r", "Q", "K1", "V1", "K2", "V2", "K3", "V3"] + (["dO"] if self.kind == "train" else [])
         if self.kind == "fuse":
             names.remove("Q")
+        if self.kind == "summary":
+            names = ["X"]
         self.t = {n: make_tensor(cfg, n, device) for n in names}
         B, H, T, d, D = cfg.B, cfg.H, cfg.T, cfg.d, cfg.D
+        if self.kind == "summary":
+            self.M2 = torch.empty_like(self.t["X"])
+            self.state = torch.zeros(B, D, device=device)
+            self.ws = torch.zeros(256, dtype=torch.uint8, device=device)
+            self.launches_per_step = 1
+            self.work = dict(self.work)
+            self.ev = []
+            return
         self.K = [self.t["K1"], self.t["K2"], self.t["K3"]]
         self.V = [self.t["V1"], self.t["V2"], self.t["V3"]]
         self.shape = mka.make_shape(B, H, T, d, D, cfg.W, 0)
@@ -172,6 +185,14 @@ class Leg:
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
         if record:
             e[0].record()
+        if self.kind == "summary":
+            if record:
+                e[1].record()
+            mka.mka_l2_summary(t["X"], mka.MKA_SUMMARY_MEAN, state=self.state, n_prev=0, M2=self.M2, ws=self.ws)
+            if record:
+                e[2].record(); e[3].record()
+                self.ev.append(e)
+            return
         mka.mka_router(t["X"], t["W_r"], None, gate=self.gate)
         if record:
             e[1].record()
@@ -192,6 +213,8 @@ class Leg:
             self.ev.append(e)
 
     def result_tensor(self):
+        if self.kind == "summary":
+            return self.M2
         if self.kind == "fuse":
             return self.cache_k
         return self.Od if self.kind == "decode" else (self.grads["dQ"] if self.kind == "train" else self.O)
@@ -228,7 +251,14 @@ def timed_steps(leg, steps, warmup, dist=None):
 
 def leg_report(leg, ms_per_step, n_gpus, peaks):
     cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
-    if leg.kind == "fuse":
+    if leg.kind == "summary":
+        achieved = w["summary_bytes"] / (k["main"] * 1e-3) / 1e9
+        roof = {"kernel": "l2_summary_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
+                "peak_source": peaks["source"], "traffic": ncu_traffic("l2_summary_kernel@s3", cfg) if leg.name[:2] == "s3" else None}
+        value = n_gpus * w["summary_bytes"] / (ms_per_step * 1e-3) / 1e9
+        unit, metric = "GB/s", "l2_summary_hbm_gbs"
+    elif leg.kind == "fuse":
         achieved = w["fuse_bytes"] / (k["main"] * 1e-3) / 1e9
         roof = {"kernel": "fuse_kv_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
@@ -335,6 +365,14 @@ def oracle_sample(name, budget_rows=None):
         bytes_ = 2.0 * 2.0 * d * sum(cfg.N) * len(heads)
         return {"value": bytes_ / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle", "seconds": dt,
                 "sample": f"{len(heads)} of {cfg.B * cfg.H} (batch, head) pairs, all {sum(cfg.N)} cached rows each"}
+    if name[:2] == "s3":
+        rows = min(cfg.T, 4096)
+        X = make_tensor(cfg, "X", flat_start=0, flat_count=rows * cfg.D).double().numpy().reshape(1, rows, cfg.D)
+        t0 = time.perf_counter()
+        orc.l2_summary(X, orc.SUMMARY_MEAN)
+        dt = time.perf_counter() - t0
+        return {"value": 2.0 * 2.0 * cfg.D * rows / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dt,
+                "sample": f"the first {rows} of {cfg.T} tokens of one sequence (numpy, one thread)"}
     if name[:2] == "f3":
         X, Wr = _router_inputs(cfg)
         t0 = time.perf_counter()
@@ -391,8 +429,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "c3p", "c4p", "c5p", "f3p"])
-    ap.add_argument("--legs", default="c4,c5,c2,f3", help="other configurations measured after the primary one ('' = none)")
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "s3", "c3p", "c4p", "c5p", "f3p", "s3p"])
+    ap.add_argument("--legs", default="c4,c5,c2,f3,s3", help="other configurations measured after the primary one ('' = none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -402,7 +440,7 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     cfg = CONFIGS[args.workload]
     wk = args.workload[:2]
-    metric_name = {"c4": "decode_hbm_gbs", "c5": "fwd_bwd_tflops", "f3": "route_fuse_hbm_gbs"}.get(wk, "prefill_fwd_tflops")
+    metric_name = {"c4": "decode_hbm_gbs", "c5": "fwd_bwd_tflops", "f3": "route_fuse_hbm_gbs", "s3": "l2_summary_hbm_gbs"}.get(wk, "prefill_fwd_tflops")
     base = {"metric": f"FastMKA {metric_name} (algorithmic, visible pairs only)", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
             "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
@@ -457,6 +495,8 @@ def main():
             ev = world * w["decode_bytes"] / (e_ms * 1e-3) / 1e9
         elif wk == "f3":
             ev = world * w["fuse_bytes"] / (e_ms * 1e-3) / 1e9
+        elif wk == "s3":
+            ev = world * w["summary_bytes"] / (e_ms * 1e-3) / 1e9
         else:
             ev = world * (w["fwd_flops"] + (w["bwd_flops"] if wk == "c5" else 0.0)) / (e_ms * 1e-3) / 1e12
         out["e2e"] = {"value": ev, "unit": rep["unit"], "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}

@@ -138,6 +138,9 @@ CONFIGS: Dict[str, WorkloadConfig] = {
     # route-fusion / cache write of Alg. 2 (levels token-aligned): c3's geometry with N_3 = T, and a profiler-sized variant
     "f3": WorkloadConfig("f3", 5, "bf16", 1, 32, 128, 4096, 32768, 4096, (32768, 32768, 32768)),
     "f3p": WorkloadConfig("f3p", 5, "bf16", 1, 8, 128, 4096, 32768, 4096, (32768, 32768, 32768)),
+    # L2 session summary (a scan over the router input X of c3), and a profiler-sized variant
+    "s3": WorkloadConfig("s3", 6, "bf16", 1, 32, 128, 4096, 32768, 4096, (32768, 32768, 8192)),
+    "s3p": WorkloadConfig("s3p", 6, "bf16", 1, 32, 128, 4096, 12288, 4096, (12288, 12288, 8192)),
     # profiler-sized variants (same per-head geometry, fewer heads / sequences) for ncu captures
     "c3p": WorkloadConfig("c3p", 2, "bf16", 1, 8, 128, 4096, 32768, 4096, (32768, 32768, 8192)),
     "c4p": WorkloadConfig("c4p", 3, "bf16", 2, 32, 128, 4096, 1, 4096, (4096, 32768, 8192), decode=True),
