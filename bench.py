@@ -56,7 +56,7 @@ NCU_TRAFFIC = {
     "fwd_tc_kernel@c3": (376.368896e6 + 67.608320e6, 1 * 8),
     "decode_partial_kernel@c4": (1.476439e9 + 6.574e6, 2 * 32),
     "bwd_dq_tc_kernel@c5": (220.280064e6 + 26.611200e6, 1 * 16),
-    "l2_summary_kernel@s3": None,
+    "l2_summary_kernel@s3": (100.742400e6 + 53.976576e6, 12288.0 / 32768.0),   # captured on 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.135744e6 + 84.349696e6, 1 * 8),
     "bwd_dkv_tc_kernel@c5": (220.329216e6 + 114.653440e6, 1 * 16),
 }
@@ -66,7 +66,8 @@ def ncu_traffic(key, cfg):
     ent = NCU_TRAFFIC.get(key)
     if ent is None:
         return None
-    return ent[0] * (cfg.B * cfg.H) / ent[1]
+    units = cfg.B if key.startswith("l2_summary") else cfg.B * cfg.H     # the summary's unit is a whole sequence
+    return ent[0] * units / ent[1]
 
 
 def algorithmic_work(cfg):
