@@ -56,7 +56,7 @@ NCU_TRAFFIC = {
     "fwd_tc_kernel@c3": (376.368896e6 + 67.608320e6, 1 * 8),
     "decode_partial_kernel@c4": (1.476439e9 + 6.574e6, 2 * 32),
     "bwd_dq_tc_kernel@c5": (220.280064e6 + 26.611200e6, 1 * 16),
-    "l2_summary_kernel@s3": (100.742400e6 + 53.976576e6, 12288.0 / 32768.0),   # captured on 12288 of the 32768 tokens
+    "l2_summary_seg_kernel@s3": (101.445120e6 + 51.656448e6, 12288.0 / 32768.0),   # captured on 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.135744e6 + 84.349696e6, 1 * 8),
     "bwd_dkv_tc_kernel@c5": (220.329216e6 + 114.653440e6, 1 * 16),
 }
@@ -148,7 +148,7 @@ class Leg:
         if self.kind == "summary":
             self.M2 = torch.empty_like(self.t["X"])
             self.state = torch.zeros(B, D, device=device)
-            self.ws = torch.zeros(256, dtype=torch.uint8, device=device)
+            self.ws = mka.mka_l2_summary_workspace(self.t["X"]).zero_()
             self.launches_per_step = 1
             self.work = dict(self.work)
             self.ev = []
@@ -254,9 +254,9 @@ def leg_report(leg, ms_per_step, n_gpus, peaks):
     cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
     if leg.kind == "summary":
         achieved = w["summary_bytes"] / (k["main"] * 1e-3) / 1e9
-        roof = {"kernel": "l2_summary_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        roof = {"kernel": "l2_summary_seg_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
-                "peak_source": peaks["source"], "traffic": ncu_traffic("l2_summary_kernel@s3", cfg) if leg.name[:2] == "s3" else None}
+                "peak_source": peaks["source"], "traffic": ncu_traffic("l2_summary_seg_kernel@s3", cfg) if leg.name[:2] == "s3" else None}
         value = n_gpus * w["summary_bytes"] / (ms_per_step * 1e-3) / 1e9
         unit, metric = "GB/s", "l2_summary_hbm_gbs"
     elif leg.kind == "fuse":

@@ -25,7 +25,7 @@ TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
-           "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_decode_static", "mka_decode_static_max_bytes"]
+           "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_l2_summary_workspace_bytes", "mka_l2_summary_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes"]
 
 
 class MkaError(RuntimeError):
@@ -84,10 +84,13 @@ def _load() -> ctypes.CDLL:
     lib.mka_decode_static_max_bytes.argtypes = []
     lib.mka_fwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level)]
     lib.mka_fuse_kv.argtypes = [i32, i32, i64, i32, i32, ctypes.POINTER(mka_level), vp, ctypes.POINTER(mka_level_grad), i64, vp]
+    lib.mka_l2_summary_workspace_bytes.restype = ctypes.c_size_t
+    lib.mka_l2_summary_workspace_bytes.argtypes = [i32, i64, i32, i32]
+    lib.mka_l2_summary_kernel_kind.argtypes = [i32, i64, i32, i32, ctypes.c_size_t]
     lib.mka_l2_summary.argtypes = [vp, i32, i64, i32, i32, i32, ctypes.c_float, vp, i64, vp, vp, ctypes.c_size_t, vp]
     lib.mka_bwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level), vp]
     for name in EXPORTS:
-        if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes"):
+        if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes", "mka_l2_summary_workspace_bytes"):
             getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -275,6 +278,18 @@ def mka_fuse_kv(K, V, gate, out_k=None, out_v=None, dst_offset=0, stream=None):
     _check(lib.mka_fuse_kv(B, H, n, d, _dt(ref), _levels(K, V), _ptr(gate), ctypes.byref(dst), dst_offset, _stream(stream)),
            "mka_fuse_kv")
     return out_k, out_v
+
+
+def mka_l2_summary_workspace(X) -> torch.Tensor:
+    """Scratch for mka_l2_summary's segmented form on input X (uint8 tensor on X's device)."""
+    B, T, D = X.shape
+    return torch.empty(int(lib.mka_l2_summary_workspace_bytes(B, T, D, _dt(X))), dtype=torch.uint8, device=X.device)
+
+
+def mka_l2_summary_kernel_kind(X, ws=None) -> int:
+    """1 when mka_l2_summary(X, ws=ws) would run the segmented form, 0 for the strip form."""
+    B, T, D = X.shape
+    return int(lib.mka_l2_summary_kernel_kind(B, T, D, _dt(X), 0 if ws is None else ws.numel()))
 
 
 def mka_l2_summary(X, kind=MKA_SUMMARY_MEAN, beta=0.9, state=None, n_prev=0, M2=None, ws=None, stream=None):

@@ -317,6 +317,20 @@ mka_status mka_fuse_kv(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype
     return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
 }
 
+size_t mka_l2_summary_workspace_bytes(int32_t B, int64_t T, int32_t D, int32_t dtype) {
+    if (B < 0 || T < 0 || D < 0 || (dtype != MKA_BF16 && dtype != MKA_F32)) return 0;
+    return kWsHeader + l2_summary_seg_workspace(B, T, D, dtype);
+}
+
+int32_t mka_l2_summary_kernel_kind(int32_t B, int64_t T, int32_t D, int32_t dtype, size_t ws_bytes) {
+    if (B <= 0 || T <= 0 || D <= 0 || (dtype != MKA_BF16 && dtype != MKA_F32)) return 0;
+    const long long strips128 = (long long)B * ((D * (dtype == MKA_BF16 ? 2 : 4) + 127) / 128);
+    // Measured: bf16 inputs gain from the segmented form at any width; fp32 rows are twice as many bytes, and the strip
+    // form already streams them well once there are about a hundred strips.
+    const bool narrow = dtype == MKA_BF16 || strips128 < 96;
+    return T >= 512 && narrow && ws_bytes >= kWsHeader + l2_summary_seg_workspace(B, T, D, dtype) ? 1 : 0;
+}
+
 mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_t dtype, int32_t kind, float beta, float* state,
                           int64_t n_prev, void* M2, void* ws, size_t ws_bytes, void* stream) {
     if (dtype != MKA_BF16 && dtype != MKA_F32) return MKA_ERR_ARG;
@@ -332,8 +346,14 @@ mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_
     if (ws && ws_bytes < kWsHeader) return MKA_ERR_WORKSPACE;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (ws && cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
-    cudaError_t e = launch_l2_summary(X, M2, state, n_prev > 0 ? 1 : 0, n_prev, B, T, D, dtype, kind, beta,
-                                      static_cast<unsigned int*>(ws), cs);
+    // With enough scratch the segmented (look-back) form cuts the sequences into 256-row segments, which keeps the GPU
+    // busy however few column strips there are; otherwise one CTA walks each strip from end to end.
+    const bool segmented = ws && (reinterpret_cast<uintptr_t>(ws) & 15) == 0 && mka_l2_summary_kernel_kind(B, T, D, dtype, ws_bytes) == 1;
+    cudaError_t e = segmented
+        ? launch_l2_summary_seg(X, M2, state, n_prev > 0 ? 1 : 0, n_prev, B, T, D, dtype, kind, beta,
+                                static_cast<unsigned int*>(ws), static_cast<char*>(ws) + kWsHeader, cs)
+        : launch_l2_summary(X, M2, state, n_prev > 0 ? 1 : 0, n_prev, B, T, D, dtype, kind, beta,
+                            static_cast<unsigned int*>(ws), cs);
     if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
     return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
 }

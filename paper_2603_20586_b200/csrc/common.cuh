@@ -123,6 +123,9 @@ cudaError_t launch_fuse_kv(const LevelDev L[3], const LevelGradDev& out, const f
                            long long dst_offset, int dtype, cudaStream_t st);
 cudaError_t launch_l2_summary(const void* X, void* M2, float* state, int use_state, long long n_prev, int B, long long T, int D,
                               int dtype, int kind, float beta, unsigned int* status, cudaStream_t st);
+size_t l2_summary_seg_workspace(int B, long long T, int D, int dtype);
+cudaError_t launch_l2_summary_seg(const void* X, void* M2, float* state, int use_state, long long n_prev, int B, long long T,
+                                  int D, int dtype, int kind, float beta, unsigned int* status, void* scratch, cudaStream_t st);
 cudaError_t launch_bwd_dgate(const float* Gpart, int B, int H, long long T, float* dG, cudaStream_t st);
 // Tensor-core (TMA + tcgen05) backward; same contract as the forward below.
 cudaError_t launch_bwd_tc(const BwdParams& p, unsigned int* status_word, cudaStream_t st);
