@@ -288,3 +288,48 @@ def l2_summary(X, kind: int = SUMMARY_MEAN, beta: float = 0.9, state=None, n_pre
             M[:, t] = m
         return M, (m if m is not None else np.zeros((B, D)))
     raise ValueError("unknown summary kind")
+
+
+def gather_pages(pool, table, rows: int, page_rows: int) -> np.ndarray:
+    """Dense view of one sequence's rows of a paged level (the paged KV layout of the paper's inference setup for
+    contexts beyond 32K).  pool is [P, H_kv, page_rows, d]; logical row r of the sequence lives in pool page
+    table[r // page_rows] at offset r % page_rows.  Returns [H_kv, rows, d].  Written row by row."""
+    pool = np.asarray(pool)
+    out = np.empty((pool.shape[1], rows, pool.shape[3]), dtype=np.float64)
+    for r in range(rows):
+        out[:, r, :] = pool[int(table[r // page_rows]), :, r % page_rows, :]
+    return out
+
+
+def decode_paged(q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, rows: Sequence, page_rows: int, gate,
+                 scale: Optional[float] = None):
+    """Single-token decode of Eq. 5 over paged levels with grouped-query sharing of the KV heads.
+
+    q [B, H, d]; for level l: pools_k[l], pools_v[l] [P_l, H_kv, page_rows, d] (or None for an absent level),
+    tables[l] [B, pages] page table, rows[l] [B] valid rows of every sequence; gate [B, 3].
+    Query head h reads KV head h // (H / H_kv): consecutive query heads share one KV head.
+    Every sequence is gathered into dense levels and handed to the dense decode (all gathered rows visible).
+    Returns O [B, H, d], LSE [B, H]."""
+    q = _f64(q)
+    gate = _f64(gate)
+    B, H, d = q.shape
+    O = np.empty((B, H, d))
+    LSE = np.empty((B, H))
+    for b in range(B):
+        Ks, Vs = [], []
+        for l in range(3):
+            if pools_k[l] is None or int(rows[l][b]) == 0:
+                Ks.append(np.zeros((1, H, 0, d)))
+                Vs.append(np.zeros((1, H, 0, d)))
+                continue
+            H_kv = np.asarray(pools_k[l]).shape[1]
+            assert H % H_kv == 0
+            kd = gather_pages(_f64(pools_k[l]), tables[l][b], int(rows[l][b]), page_rows)
+            vd = gather_pages(_f64(pools_v[l]), tables[l][b], int(rows[l][b]), page_rows)
+            share = np.arange(H) // (H // H_kv)                  # KV head of every query head
+            Ks.append(kd[share][None])
+            Vs.append(vd[share][None])
+        o, ls = fwd(q[b][None, :, None, :], Ks, Vs, gate[b].reshape(1, 1, 3), 1, scale=scale, decode=True)
+        O[b] = o[0, :, 0, :]
+        LSE[b] = ls[0, :, 0]
+    return O, LSE
