@@ -156,6 +156,34 @@ mka_status mka_fwd(const mka_shape* shape, const void* Q, const mka_level L[3], 
 mka_status mka_decode(const mka_shape* shape, const void* q, const mka_level L[3], const float* gate,
                       void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
 
+/* One memory level kept in PAGES (the paged KV layout the paper's inference setup uses for contexts beyond 32K):
+ * pools k, v hold fixed-size pages; element (page, kv head, row, :) sits at page*stride_page + head*stride_h +
+ * row*stride_n (ELEMENTS, d contiguous).  Logical row r of sequence b is row r % page_rows of pool page
+ * page_table[b*table_stride + r / page_rows].  n may be 0 (then the pointers may be NULL). */
+typedef struct mka_paged_level {
+    const void *k, *v;          /* device, bf16 */
+    const int32_t* page_table;  /* device [B, table_stride]; entries of pages that hold no valid row are never read */
+    const int32_t* rows;        /* device [B]: valid rows of every sequence (clamped to [0, n]), or NULL = n for all */
+    int64_t n;                  /* upper bound of the sequences' rows (host); table_stride * page_rows >= n */
+    int64_t table_stride;
+    int32_t page_rows;          /* rows per page: a power of two */
+    int64_t stride_page, stride_h, stride_n;
+} mka_paged_level;
+
+/*
+ * Split-KV single-token decode over paged levels with grouped-query sharing of the KV heads (the paper evaluates on
+ * GQA models and serves long contexts from a paged KV cache; Eq. 5 itself is unchanged): same result as mka_decode on
+ * the gathered, head-repeated levels.  shape->H query heads share H_kv KV heads, consecutive query heads one KV head
+ * (head h reads KV head h / (H / H_kv)); H must be a multiple of H_kv with at most 16 query heads per KV head.
+ * Every cached row is read once per KV head.  A level whose gate is exactly 0 for a sequence is not read.
+ *   q [B, H, d] bf16;  gate [B, 3] f32;  O [B, H, d] bf16;  LSE [B, H] f32 or NULL
+ *   ws: mka_decode_paged_workspace_bytes(shape, H_kv, n_level) bytes, n_level[l] = L[l].n
+ * d must be 64 or 128; pools 16-byte aligned with strides that are multiples of 8 elements.
+ */
+size_t mka_decode_paged_workspace_bytes(const mka_shape* shape, int32_t H_kv, const int64_t n_level[3]);
+mka_status mka_decode_paged(const mka_shape* shape, int32_t H_kv, const void* q, const mka_paged_level L[3],
+                            const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
+
 /*
  * Backward of mka_fwd in MKA_MODE_FAST (derived from Eq. 5; the paper prints no backward).  With
  * p = lambda exp(s - LSE) on the visible set and D_t = dO_t . O_t:

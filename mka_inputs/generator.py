@@ -163,3 +163,76 @@ def make_tensor(cfg: WorkloadConfig, name: str, device="cpu", flat_start: int = 
         return approx_normal(cfg.seed, TENSOR_IDS[name], 0, total, std, device, dtype).view(shape)
     assert 0 <= flat_start and flat_start + flat_count <= total
     return approx_normal(cfg.seed, TENSOR_IDS[name], flat_start, flat_count, std, device, dtype)
+
+
+# ---- paged levels (serving layout): page pools plus per-sequence page tables -------------------------------------------
+
+@dataclass(frozen=True)
+class PagedConfig:
+    """A paged, grouped-query decode workload: B sequences, H query heads sharing H_kv KV heads of width d, levels of
+    N rows at most, kept in pages of page_rows rows.  `rows_frac[b % len]` scales every level's rows for sequence b
+    (a mix of lengths); `spare` extra pages per pool are never referenced."""
+    name: str
+    seed: int
+    B: int
+    H: int
+    H_kv: int
+    d: int
+    N: Tuple[int, int, int]
+    page_rows: int
+    rows_frac: Tuple[float, ...] = (1.0,)
+    spare: int = 3
+
+
+PAGED_CONFIGS: Dict[str, PagedConfig] = {
+    # Qwen2.5-7B-like head geometry (28 query heads on 4 KV heads), a 128K-token session level
+    "g4": PagedConfig("g4", 7, 4, 28, 4, 128, (4096, 131072, 8192), 16),
+    "g4p": PagedConfig("g4p", 7, 1, 28, 4, 128, (4096, 131072, 8192), 16),
+    "g1": PagedConfig("g1", 8, 3, 12, 4, 64, (100, 700, 333), 16, rows_frac=(1.0, 0.37, 0.0)),
+}
+
+
+def paged_rows(cfg: PagedConfig):
+    """int32 [3][B]: valid rows of every sequence on every level."""
+    out = []
+    for l in range(3):
+        out.append(torch.tensor([int(cfg.N[l] * cfg.rows_frac[b % len(cfg.rows_frac)]) for b in range(cfg.B)],
+                                dtype=torch.int32))
+    return out
+
+
+def paged_tables(cfg: PagedConfig):
+    """Page tables int32 [3][B, pages] and pool sizes: the pages a sequence needs are dealt from a seeded shuffle of the
+    pool, so consecutive logical pages are scattered; table entries past a sequence's last page are 0."""
+    rows = paged_rows(cfg)
+    tables, pool_pages = [], []
+    for l in range(3):
+        per_seq = [-(-int(r) // cfg.page_rows) for r in rows[l]]
+        width = max(1, -(-cfg.N[l] // cfg.page_rows))
+        P = sum(per_seq) + cfg.spare
+        gen = torch.Generator().manual_seed(cfg.seed * 1000 + l)
+        order = torch.randperm(P, generator=gen).to(torch.int32)
+        tab = torch.zeros(cfg.B, width, dtype=torch.int32)
+        nxt = 0
+        for b in range(cfg.B):
+            tab[b, :per_seq[b]] = order[nxt:nxt + per_seq[b]]
+            nxt += per_seq[b]
+        tables.append(tab)
+        pool_pages.append(P)
+    return tables, pool_pages
+
+
+def make_paged(cfg: PagedConfig, device="cpu"):
+    """q [B, H, d], pools_k / pools_v [3][P_l, H_kv, page_rows, d] (bf16), tables, rows, gate logits source X-free:
+    the gate itself is drawn as three positive numbers per sequence, normalised by the caller."""
+    tables, pool_pages = paged_tables(cfg)
+    q = approx_normal(cfg.seed, 20, 0, cfg.B * cfg.H * cfg.d, 1.0, device, torch.bfloat16).view(cfg.B, cfg.H, cfg.d)
+    pk, pv = [], []
+    for l in range(3):
+        shape = (pool_pages[l], cfg.H_kv, cfg.page_rows, cfg.d)
+        cnt = shape[0] * shape[1] * shape[2] * shape[3]
+        pk.append(approx_normal(cfg.seed, 21 + 2 * l, 0, cnt, 1.0, device, torch.bfloat16).view(shape))
+        pv.append(approx_normal(cfg.seed, 22 + 2 * l, 0, cnt, 1.0, device, torch.bfloat16).view(shape))
+    g = approx_normal(cfg.seed, 27, 0, cfg.B * 3, 1.0, device, torch.float32).view(cfg.B, 3).abs() + 0.05
+    return {"q": q, "pools_k": pk, "pools_v": pv, "tables": [t.to(device) for t in tables],
+            "rows": [r.to(device) for r in paged_rows(cfg)], "gate_raw": g}

@@ -25,7 +25,8 @@ TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
-           "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_l2_summary_workspace_bytes", "mka_l2_summary_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes"]
+           "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_l2_summary_workspace_bytes", "mka_l2_summary_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes",
+           "mka_decode_paged", "mka_decode_paged_workspace_bytes"]
 
 
 class MkaError(RuntimeError):
@@ -42,6 +43,13 @@ class mka_level(ctypes.Structure):
 class mka_level_grad(ctypes.Structure):
     _fields_ = [("dk", ctypes.c_void_p), ("dv", ctypes.c_void_p), ("n", ctypes.c_int64),
                 ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64)]
+
+
+class mka_paged_level(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("page_table", ctypes.c_void_p),
+                ("rows", ctypes.c_void_p), ("n", ctypes.c_int64), ("table_stride", ctypes.c_int64),
+                ("page_rows", ctypes.c_int32), ("stride_page", ctypes.c_int64), ("stride_h", ctypes.c_int64),
+                ("stride_n", ctypes.c_int64)]
 
 
 class mka_shape(ctypes.Structure):
@@ -86,11 +94,16 @@ def _load() -> ctypes.CDLL:
     lib.mka_fuse_kv.argtypes = [i32, i32, i64, i32, i32, ctypes.POINTER(mka_level), vp, ctypes.POINTER(mka_level_grad), i64, vp]
     lib.mka_l2_summary_workspace_bytes.restype = ctypes.c_size_t
     lib.mka_l2_summary_workspace_bytes.argtypes = [i32, i64, i32, i32]
+    lib.mka_decode_paged_workspace_bytes.restype = ctypes.c_size_t
+    lib.mka_decode_paged_workspace_bytes.argtypes = [ctypes.POINTER(mka_shape), i32, ctypes.POINTER(ctypes.c_int64)]
+    lib.mka_decode_paged.argtypes = [ctypes.POINTER(mka_shape), i32, vp, ctypes.POINTER(mka_paged_level), vp, vp, vp, vp,
+                                     ctypes.c_size_t, vp]
     lib.mka_l2_summary_kernel_kind.argtypes = [i32, i64, i32, i32, ctypes.c_size_t]
     lib.mka_l2_summary.argtypes = [vp, i32, i64, i32, i32, i32, ctypes.c_float, vp, i64, vp, vp, ctypes.c_size_t, vp]
     lib.mka_bwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level), vp]
     for name in EXPORTS:
-        if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes", "mka_l2_summary_workspace_bytes"):
+        if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes", "mka_l2_summary_workspace_bytes",
+                        "mka_decode_paged_workspace_bytes"):
             getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -206,6 +219,41 @@ def mka_decode(shape: mka_shape, q, K, V, gate, O=None, LSE=None, ws=None, strea
         ws = alloc_workspace(shape, n, MKA_WS_DECODE, q.device)
     _check(lib.mka_decode(ctypes.byref(shape), _ptr(q), _levels(K, V), _ptr(gate), _ptr(O), _ptr(LSE), _ptr(ws),
                           ws.numel(), _stream(stream)), "mka_decode")
+    return O, LSE
+
+
+def _paged_levels(pools_k, pools_v, tables, rows, n):
+    arr = (mka_paged_level * 3)()
+    for l in range(3):
+        k, v = pools_k[l], pools_v[l]
+        if k is None or n[l] == 0:
+            arr[l] = mka_paged_level(None, None, None, None, 0, 0, 1, 0, 0, 0)
+            continue
+        # pools [pages, H_kv, page_rows, d]; any strides with d contiguous
+        assert k.dim() == 4 and k.stride(3) == 1 and v.stride() == k.stride() and v.shape == k.shape
+        tab = tables[l]
+        assert tab.dtype == torch.int32 and tab.dim() == 2 and tab.stride(1) == 1
+        r = None if rows is None else rows[l]
+        assert r is None or (r.dtype == torch.int32 and r.is_contiguous())
+        arr[l] = mka_paged_level(k.data_ptr(), v.data_ptr(), tab.data_ptr(), _ptr(r), int(n[l]), tab.stride(0),
+                                 k.shape[2], k.stride(0), k.stride(1), k.stride(2))
+    return arr
+
+
+def mka_decode_paged(shape: mka_shape, H_kv: int, q, pools_k, pools_v, tables, n, gate, rows=None, O=None, LSE=None,
+                     ws=None, stream=None):
+    """Decode over paged levels with grouped-query head sharing.  pools_k[l], pools_v[l]: [pages, H_kv, page_rows, d]
+    (or None); tables[l]: int32 [B, pages per sequence]; n[l]: upper bound of the rows; rows[l]: int32 [B] or None."""
+    assert q.is_contiguous() and gate.is_contiguous() and gate.dtype == torch.float32
+    if O is None:
+        O = torch.empty_like(q)
+    if LSE is None:
+        LSE = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    if ws is None:
+        ws = torch.empty(int(lib.mka_decode_paged_workspace_bytes(ctypes.byref(shape), H_kv, _n_level(n))),
+                         dtype=torch.uint8, device=q.device)
+    _check(lib.mka_decode_paged(ctypes.byref(shape), H_kv, _ptr(q), _paged_levels(pools_k, pools_v, tables, rows, n),
+                                _ptr(gate), _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream)), "mka_decode_paged")
     return O, LSE
 
 

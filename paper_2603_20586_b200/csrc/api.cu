@@ -222,6 +222,68 @@ mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], c
     return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
 }
 
+size_t mka_decode_paged_workspace_bytes(const mka_shape* s, int32_t H_kv, const int64_t n_level[3]) {
+    if (!s || !n_level || H_kv <= 0 || s->B < 0 || s->H < 0 || s->d <= 0) return 0;
+    mka_decode_plan_t plan;
+    if (mka_decode_plan(n_level, s->B, H_kv, s->d, &plan) != MKA_OK) return 0;
+    return kWsHeader + round_up((size_t)s->B * s->H * plan.total_chunks * (s->d + 2) * sizeof(float), 256);
+}
+
+mka_status mka_decode_paged(const mka_shape* s, int32_t H_kv, const void* q, const mka_paged_level L[3],
+                            const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream) {
+    mka_status st = check_shape(s, true);
+    if (st != MKA_OK) return st;
+    if (s->dtype != MKA_BF16 || s->mode != MKA_MODE_FAST) return MKA_ERR_UNSUPPORTED;
+    if (s->d != 64 && s->d != 128) return MKA_ERR_SHAPE;
+    if (!L) return MKA_ERR_ARG;
+    if (H_kv <= 0 || (s->H > 0 && (s->H % H_kv != 0 || s->H / H_kv > 16))) return MKA_ERR_SHAPE;
+    int64_t n_level[3];
+    DecodePagedParams p;
+    memset(&p, 0, sizeof(p));
+    for (int l = 0; l < 3; ++l) {
+        n_level[l] = L[l].n;
+        if (L[l].n < 0) return MKA_ERR_SHAPE;
+        if (L[l].n == 0) continue;
+        if (!L[l].k || !L[l].v || !L[l].page_table) return MKA_ERR_ARG;
+        const int pr = L[l].page_rows;
+        if (pr <= 0 || (pr & (pr - 1)) != 0) return MKA_ERR_SHAPE;
+        if (L[l].table_stride * pr < L[l].n) return MKA_ERR_SHAPE;
+        if (L[l].stride_n < s->d || L[l].stride_page < 0 || L[l].stride_h < 0) return MKA_ERR_SHAPE;
+        if (!aligned16(L[l].k) || !aligned16(L[l].v)) return MKA_ERR_ALIGN;
+        if (L[l].stride_n % 8 || L[l].stride_page % 8 || L[l].stride_h % 8) return MKA_ERR_ALIGN;
+        int shift = 0;
+        while ((1 << shift) < pr) ++shift;
+        p.L[l].k = L[l].k; p.L[l].v = L[l].v; p.L[l].table = L[l].page_table; p.L[l].rows = L[l].rows;
+        p.L[l].n = L[l].n; p.L[l].table_stride = L[l].table_stride;
+        p.L[l].sp = L[l].stride_page; p.L[l].sh = L[l].stride_h; p.L[l].sn = L[l].stride_n;
+        p.L[l].page_shift = shift;
+    }
+    if (s->B == 0 || s->H == 0) return MKA_OK;
+    if (!q || !gate || !O) return MKA_ERR_ARG;
+    if (!aligned16(q) || !aligned16(O)) return MKA_ERR_ALIGN;
+    const size_t need = mka_decode_paged_workspace_bytes(s, H_kv, n_level);
+    if (!ws || ws_bytes < need) return MKA_ERR_WORKSPACE;
+    mka_decode_plan_t plan;
+    mka_decode_plan(n_level, s->B, H_kv, s->d, &plan);
+    if ((long long)s->B * s->H * plan.total_chunks > 0x7fffffffLL) return MKA_ERR_SHAPE;
+    p.q = q; p.gate = gate;
+    p.B = s->B; p.H = s->H; p.H_kv = H_kv; p.d = s->d; p.scale = resolve_scale(s);
+    p.chunk_rows = plan.chunk_rows;
+    p.total_chunks = plan.total_chunks;
+    p.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeader);
+    DecodeParams c;                                    // the combine kernel of the dense decode finishes the job
+    memset(&c, 0, sizeof(c));
+    c.O = O; c.LSE = LSE; c.gate = gate; c.B = s->B; c.H = s->H; c.d = s->d;
+    c.total_chunks = plan.total_chunks; c.partial = p.partial;
+    for (int l = 0; l < 3; ++l) { p.n_chunks[l] = plan.n_chunks[l]; c.n_chunks[l] = plan.n_chunks[l]; }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
+    cudaError_t e = launch_decode_paged(p, cs);
+    if (e == cudaSuccess) e = launch_decode_combine(c, cs);
+    if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
 mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], const float* gate, const void* O,
                    const float* LSE, const void* dO, const void* R, int32_t r_dtype, void* dQ,
                    const mka_level_grad dL[3], float* dG, float* dW_r, float* db_r, void* ws, size_t ws_bytes,

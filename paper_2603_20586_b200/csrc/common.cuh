@@ -99,6 +99,28 @@ struct DecodeParams {
     float* partial;      // [B*H, total_chunks, d+2]
 };
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st);
+cudaError_t launch_decode_combine(const DecodeParams& p, cudaStream_t st);   // second kernel alone (gate, n_chunks, partial, O, LSE)
+
+struct PagedLevelDev {
+    const void* k;
+    const void* v;
+    const int* table;    // [B, table_stride]
+    const int* rows;     // [B] or null
+    long long n, table_stride, sp, sh, sn;
+    int page_shift;      // log2(page_rows)
+};
+struct DecodePagedParams {
+    const void* q;
+    const float* gate;   // [B,3]
+    PagedLevelDev L[3];
+    int B, H, H_kv, d;
+    float scale;
+    long long chunk_rows;
+    long long n_chunks[3];
+    long long total_chunks;
+    float* partial;      // [B*H, total_chunks, d+2]
+};
+cudaError_t launch_decode_paged(const DecodePagedParams& p, cudaStream_t st);
 
 struct BwdParams {
     const void *Q, *O, *dO;

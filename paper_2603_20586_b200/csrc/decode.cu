@@ -48,6 +48,11 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_partial_kernel(const De
     const int b = (int)(bh / p.H), h = (int)(bh % p.H);
     const long long r_begin = chunk * p.chunk_rows;
     const long long r_end = r_begin + p.chunk_rows < L.n ? r_begin + p.chunk_rows : L.n;
+    if (p.gate[b * 3 + lvl] == 0.f) {                  // hard routing switched this level off: do not read it
+        float* out = p.partial + (long long)blockIdx.x * (DH + 2);
+        for (int i = threadIdx.x; i < DH + 2; i += kWarps * 32) out[i] = i == 0 ? -INFINITY : 0.f;
+        return;
+    }
     const __nv_bfloat16* Kp = static_cast<const __nv_bfloat16*>(L.k) + b * L.sb + h * L.sh + sub * 8;
     const __nv_bfloat16* Vp = static_cast<const __nv_bfloat16*>(L.v) + b * L.sb + h * L.sh + sub * 8;
 
@@ -210,6 +215,15 @@ cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
 }
 
 }  // namespace
+
+cudaError_t launch_decode_combine(const DecodeParams& p, cudaStream_t st) {
+    const long long bh = (long long)p.B * p.H;
+    if (bh == 0) return cudaSuccess;
+    if (p.d == 128) decode_combine_kernel<128><<<(unsigned)bh, 128, 0, st>>>(p);
+    else if (p.d == 64) decode_combine_kernel<64><<<(unsigned)bh, 64, 0, st>>>(p);
+    else return cudaErrorNotSupported;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st) {
     if (p.d == 128) return launch_t<128>(p, st);
