@@ -31,7 +31,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from mka_inputs import CONFIGS, make_tensor  # noqa: E402
+from mka_inputs import CONFIGS, PAGED_CONFIGS, make_paged, make_tensor  # noqa: E402
 
 DATASHEET = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
@@ -58,6 +58,7 @@ NCU_TRAFFIC = {
     "bwd_dq_tc_kernel@c5": (220.280064e6 + 26.611200e6, 1 * 16),
     "l2_summary_seg_kernel@s3": (101.445120e6 + 51.656448e6, 12288.0 / 32768.0),   # captured on 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.135744e6 + 84.349696e6, 1 * 8),
+    "decode_paged_kernel@g4": None,        # the kernel has changed since its counters were taken
     "bwd_dkv_tc_kernel@c5": (220.329216e6 + 114.653440e6, 1 * 16),
 }
 
@@ -66,7 +67,10 @@ def ncu_traffic(key, cfg):
     ent = NCU_TRAFFIC.get(key)
     if ent is None:
         return None
-    units = cfg.B if key.startswith("l2_summary") else cfg.B * cfg.H     # the summary's unit is a whole sequence
+    if key.startswith("decode_paged"):
+        units = cfg.B * cfg.H_kv                                           # one KV head of one sequence
+    else:
+        units = cfg.B if key.startswith("l2_summary") else cfg.B * cfg.H     # the summary's unit is a whole sequence
     return ent[0] * units / ent[1]
 
 
@@ -132,6 +136,9 @@ class Leg:
     def __init__(self, name, device, seed_shift=0):
         import paper_2603_20586_b200 as mka
         self.mka, self.name, self.dev = mka, name, device
+        if name in PAGED_CONFIGS:
+            self._init_paged(PAGED_CONFIGS[name], device, seed_shift)
+            return
         cfg = CONFIGS[name]
         if seed_shift:
             cfg = type(cfg)(**{**cfg.__dict__, "seed": cfg.seed + 1000 * seed_shift})
@@ -181,8 +188,43 @@ class Leg:
             self.launches_per_step = 2              # router, fwd
         self.ev = []
 
+    def _init_paged(self, cfg, device, seed_shift):
+        """Paged, grouped-query decode: pools, page tables and the gate are resident; one step = partial + combine."""
+        import dataclasses
+        mka = self.mka
+        if seed_shift:
+            cfg = dataclasses.replace(cfg, seed=cfg.seed + 1000 * seed_shift)
+        self.cfg, self.kind = cfg, "paged"
+        P = make_paged(cfg, device)
+        self.t = {"q": P["q"]}
+        for l in range(3):
+            self.t[f"pk{l}"], self.t[f"pv{l}"] = P["pools_k"][l], P["pools_v"][l]
+        self.tables, self.rows = P["tables"], P["rows"]
+        self.gate_d = (P["gate_raw"] / P["gate_raw"].sum(1, keepdim=True)).contiguous()
+        self.shape = mka.make_shape(cfg.B, cfg.H, 1, cfg.d, 32)
+        self.Od = torch.empty_like(P["q"])
+        self.LSEd = torch.empty(cfg.B, cfg.H, device=device)
+        self.ws = torch.zeros(mka.mka_decode_paged_workspace_bytes(self.shape, cfg.H_kv, list(cfg.N)), dtype=torch.uint8,
+                              device=device)
+        rows_total = float(sum(int(r.sum()) for r in self.rows))
+        # every valid cached row of every KV head once: K and V, 2 bytes per element
+        self.work = {"decode_bytes": 2.0 * 2.0 * cfg.d * rows_total * cfg.H_kv}
+        self.launches_per_step = 2
+        self.ev = []
+
     def step(self, record=False):
         mka, t = self.mka, self.t
+        if self.kind == "paged":
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
+            if record:
+                e[0].record(); e[1].record()
+            cfg = self.cfg
+            mka.mka_decode_paged(self.shape, cfg.H_kv, t["q"], [t["pk0"], t["pk1"], t["pk2"]], [t["pv0"], t["pv1"], t["pv2"]],
+                                 self.tables, list(cfg.N), self.gate_d, rows=self.rows, O=self.Od, LSE=self.LSEd, ws=self.ws)
+            if record:
+                e[2].record(); e[3].record()
+                self.ev.append(e)
+            return
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
         if record:
             e[0].record()
@@ -214,6 +256,8 @@ class Leg:
             self.ev.append(e)
 
     def result_tensor(self):
+        if self.kind == "paged":
+            return self.Od
         if self.kind == "summary":
             return self.M2
         if self.kind == "fuse":
@@ -252,7 +296,15 @@ def timed_steps(leg, steps, warmup, dist=None):
 
 def leg_report(leg, ms_per_step, n_gpus, peaks):
     cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
-    if leg.kind == "summary":
+    if leg.kind == "paged":
+        achieved = w["decode_bytes"] / (k["main"] * 1e-3) / 1e9
+        roof = {"kernel": "decode_paged_kernel+decode_combine_kernel", "bound": "hbm", "achieved": achieved,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "frac_datasheet": achieved / DATASHEET["hbm_gbs"], "peak_source": peaks["source"],
+                "traffic": ncu_traffic("decode_paged_kernel@g4", cfg) if leg.name[:2] == "g4" else None}
+        value = n_gpus * w["decode_bytes"] / (ms_per_step * 1e-3) / 1e9
+        unit, metric = "GB/s", "decode_paged_hbm_gbs"
+    elif leg.kind == "summary":
         achieved = w["summary_bytes"] / (k["main"] * 1e-3) / 1e9
         roof = {"kernel": "l2_summary_seg_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
@@ -339,7 +391,27 @@ def _router_inputs(cfg):
     return _ROUTER_INPUTS[cfg.name]
 
 
+def oracle_sample_paged(name):
+    """The oracle's paged decode on sequence 0 of the configuration (all heads, all rows)."""
+    import dataclasses
+    from oracle import mka_oracle as orc
+    cfg = dataclasses.replace(PAGED_CONFIGS[name], B=1)
+    P = make_paged(cfg, "cpu")
+    f = lambda t: t.double().numpy()
+    gate = f(P["gate_raw"] / P["gate_raw"].sum(1, keepdim=True))
+    rows = [r.numpy().astype(np.int64) for r in P["rows"]]
+    t0 = time.perf_counter()
+    orc.decode_paged(f(P["q"]), [f(k) for k in P["pools_k"]], [f(v) for v in P["pools_v"]],
+                     [t.numpy().astype(np.int64) for t in P["tables"]], rows, cfg.page_rows, gate)
+    dt = time.perf_counter() - t0
+    bytes_ = 2.0 * 2.0 * cfg.d * float(sum(int(r.sum()) for r in rows)) * cfg.H_kv
+    return {"value": bytes_ / dt / 1e9, "unit": "GB/s", "cores": orc.num_threads(), "kind": "oracle", "seconds": dt,
+            "sample": f"one sequence of the configuration's {PAGED_CONFIGS[name].B}: all {cfg.H} heads, all {int(sum(int(r.sum()) for r in rows))} cached rows"}
+
+
 def oracle_sample(name, budget_rows=None):
+    if name in PAGED_CONFIGS:
+        return oracle_sample_paged(name)
     """Times the CPU oracle, as it stands, on a bounded seeded sample of workload `name`."""
     from oracle import mka_oracle as orc
     orc.build()
@@ -430,8 +502,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "s3", "c3p", "c4p", "c5p", "f3p", "s3p"])
-    ap.add_argument("--legs", default="c4,c5,c2,f3,s3", help="other configurations measured after the primary one ('' = none)")
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "s3", "g4", "c3p", "c4p", "c5p", "f3p", "s3p", "g4p"])
+    ap.add_argument("--legs", default="c4,c5,c2,f3,s3,g4", help="other configurations measured after the primary one ('' = none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -439,13 +511,18 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    cfg = CONFIGS[args.workload]
     wk = args.workload[:2]
-    metric_name = {"c4": "decode_hbm_gbs", "c5": "fwd_bwd_tflops", "f3": "route_fuse_hbm_gbs", "s3": "l2_summary_hbm_gbs"}.get(wk, "prefill_fwd_tflops")
+    paged = args.workload in PAGED_CONFIGS
+    cfg = PAGED_CONFIGS[args.workload] if paged else CONFIGS[args.workload]
+    metric_name = {"c4": "decode_hbm_gbs", "c5": "fwd_bwd_tflops", "f3": "route_fuse_hbm_gbs", "s3": "l2_summary_hbm_gbs",
+                   "g4": "decode_paged_hbm_gbs"}.get(wk, "prefill_fwd_tflops")
+    describe = (f"{args.workload}: B={cfg.B} H={cfg.H} H_kv={cfg.H_kv} d={cfg.d} N={list(cfg.N)} page_rows={cfg.page_rows} seed={cfg.seed}"
+                if paged else
+                f"{args.workload}: B={cfg.B} H={cfg.H} d={cfg.d} D={cfg.D} T={cfg.T} W={cfg.W} N={list(cfg.N)} seed={cfg.seed}")
     base = {"metric": f"FastMKA {metric_name} (algorithmic, visible pairs only)", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
-            "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
-            "config": {"workload": f"{args.workload}: B={cfg.B} H={cfg.H} d={cfg.d} D={cfg.D} T={cfg.T} W={cfg.W} N={list(cfg.N)} seed={cfg.seed}",
+            "dtype": "bf16" if (paged or cfg.dtype == "bf16") else "f32",
+            "config": {"workload": describe,
                        "l2": "inputs larger than L2 (no flush needed)" if args.workload != "c2" else "inputs ~235 MB, larger than the 126 MB L2",
                        "per_gpu": "each rank runs the whole configuration on its own seeded batch (no collective on the data path)"}}
 
@@ -492,7 +569,7 @@ def main():
     if not args.no_e2e:
         e_ms, h2d, d2h = e2e_run(leg, max(2, min(args.steps, 5)), 1)
         w = leg.work
-        if wk == "c4":
+        if wk in ("c4", "g4"):
             ev = world * w["decode_bytes"] / (e_ms * 1e-3) / 1e9
         elif wk == "f3":
             ev = world * w["fuse_bytes"] / (e_ms * 1e-3) / 1e9

@@ -240,6 +240,10 @@ def _paged_levels(pools_k, pools_v, tables, rows, n):
     return arr
 
 
+def mka_decode_paged_workspace_bytes(shape: mka_shape, H_kv: int, n) -> int:
+    return int(lib.mka_decode_paged_workspace_bytes(ctypes.byref(shape), H_kv, _n_level(n)))
+
+
 def mka_decode_paged(shape: mka_shape, H_kv: int, q, pools_k, pools_v, tables, n, gate, rows=None, O=None, LSE=None,
                      ws=None, stream=None):
     """Decode over paged levels with grouped-query head sharing.  pools_k[l], pools_v[l]: [pages, H_kv, page_rows, d]
@@ -250,8 +254,7 @@ def mka_decode_paged(shape: mka_shape, H_kv: int, q, pools_k, pools_v, tables, n
     if LSE is None:
         LSE = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
     if ws is None:
-        ws = torch.empty(int(lib.mka_decode_paged_workspace_bytes(ctypes.byref(shape), H_kv, _n_level(n))),
-                         dtype=torch.uint8, device=q.device)
+        ws = torch.empty(mka_decode_paged_workspace_bytes(shape, H_kv, n), dtype=torch.uint8, device=q.device)
     _check(lib.mka_decode_paged(ctypes.byref(shape), H_kv, _ptr(q), _paged_levels(pools_k, pools_v, tables, rows, n),
                                 _ptr(gate), _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream)), "mka_decode_paged")
     return O, LSE

@@ -185,17 +185,43 @@ __global__ void __launch_bounds__(DH) decode_combine_kernel(const DecodeParams p
 #pragma unroll
     for (int w = 1; w < DH / 32; ++w) M = fmaxf(M, sm[w]);
 
+    // Weights of a batch of DH chunks are worked out side by side (one chunk per thread) and parked in shared
+    // memory; the accumulation over the batch then runs without a branch, its loads independent of each other.
     float Z = 0.f, A = 0.f;
+    __shared__ float sw[DH];
     if (M > -INFINITY) {
-        for (long long c = 0; c < p.total_chunks; ++c) {
-            const float g = c < c1 ? lam[0] : (c < c2 ? lam[1] : lam[2]);
-            const float mc = part[c * (DH + 2)], zc = part[c * (DH + 2) + 1];
-            if (!(g > 0.f && zc > 0.f)) continue;
-            const float w = g * exp2f(mc - M);
-            Z = fmaf(w, zc, Z);
-            A = fmaf(w, part[c * (DH + 2) + 2 + tid], A);
+        for (long long c0 = 0; c0 < p.total_chunks; c0 += DH) {
+            const long long c = c0 + tid;
+            float w = 0.f;
+            if (c < p.total_chunks) {
+                const float g = c < c1 ? lam[0] : (c < c2 ? lam[1] : lam[2]);
+                const float mc = part[c * (DH + 2)], zc = part[c * (DH + 2) + 1];
+                if (g > 0.f && zc > 0.f) { w = g * exp2f(mc - M); Z = fmaf(w, zc, Z); }
+            }
+            __syncthreads();                                   // the previous batch has been consumed
+            sw[tid] = w;
+            __syncthreads();
+            const int nb = p.total_chunks - c0 < DH ? (int)(p.total_chunks - c0) : DH;
+            const float* col = part + c0 * (DH + 2) + 2 + tid;
+            int j = 0;
+            for (; j + 8 <= nb; j += 8) {
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = col[(long long)(j + u) * (DH + 2)];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) A = fmaf(sw[j + u], v[u], A);
+            }
+            for (; j < nb; ++j) A = fmaf(sw[j], col[(long long)j * (DH + 2)], A);
         }
     }
+    // Z: every thread holds the share of its own chunks
+    Z = warp_sum(Z);
+    __shared__ float sz[DH / 32];
+    if (lane == 0) sz[warp] = Z;
+    __syncthreads();
+    Z = 0.f;
+#pragma unroll
+    for (int w = 0; w < DH / 32; ++w) Z += sz[w];
     __nv_bfloat16* O = static_cast<__nv_bfloat16*>(p.O) + bh * DH;
     O[tid] = __float2bfloat16_rn(Z > 0.f ? A / Z : 0.f);
     if (p.LSE && tid == 0) p.LSE[bh] = Z > 0.f ? (M + log2f(Z)) * kLn2 : -INFINITY;
