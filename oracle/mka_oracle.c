@@ -345,3 +345,64 @@ int orc_bwd_head(const double *Q, int64_t T, int64_t d,
     }
     return 0;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * L3 recall (Alg. 2 step 4, "L3 <- Retrieve(Q_h)"; the method section's "vectorized hashing" with
+ * "chunk-based recall"; R = 8 recalled chunks in the passkey table).  The paper names the mechanism
+ * but not the hash, so this is a READING: every chunk of the long-term bank carries a
+ * sign-random-projection code of the sum of its keys, the query carries the code of the sum of the
+ * query heads that share the KV head, and the R chunks whose codes agree with the query's in the
+ * most bits are recalled (ties go to the earlier chunk), listed in bank order.
+ * The code bits are decided by fp32 arithmetic, so the order of that arithmetic is part of the
+ * definition: sums run row by row in fp32, projections are one fmaf chain over the columns.
+ */
+#include <stdint.h>
+
+/* s[i] = ((x[0][i] + x[1][i]) + x[2][i]) + ... in fp32 */
+int orc_sum_rows_f32(const float *x, int64_t n, int64_t d, float *s) {
+    for (int64_t i = 0; i < d; ++i) {
+        float acc = 0.0f;
+        for (int64_t r = 0; r < n; ++r) acc = acc + x[r * d + i];
+        s[i] = acc;
+    }
+    return 0;
+}
+
+/* bit j of the code = [ fmaf(P[j][d-1], x[d-1], ... fmaf(P[j][0], x[0], 0)) >= 0 ]; bits is a multiple of 32 */
+int orc_srp_code(const float *x, const float *proj, int64_t d, int64_t bits, uint32_t *code) {
+    if (bits % 32) return 1;
+    for (int64_t w = 0; w < bits / 32; ++w) code[w] = 0u;
+    for (int64_t j = 0; j < bits; ++j) {
+        float acc = 0.0f;
+        for (int64_t i = 0; i < d; ++i) acc = fmaf(proj[j * d + i], x[i], acc);
+        if (acc >= 0.0f) code[j / 32] |= 1u << (j % 32);
+    }
+    return 0;
+}
+
+/* The R entries of codes[n][words] closest to qcode in Hamming distance, ties to the lower index; their indices
+ * ascending in out[0..*n_out), *n_out = min(R, n).  Selection by repeated scan, as plain as it gets. */
+int orc_l3_select(const uint32_t *qcode, const uint32_t *codes, int64_t n, int64_t words, int64_t R, int64_t *out,
+                  int64_t *n_out) {
+    int64_t k = R < n ? R : n;
+    char *taken = (char *)calloc((size_t)(n > 0 ? n : 1), 1);
+    if (!taken) return 1;
+    for (int64_t s = 0; s < k; ++s) {
+        int64_t best = -1, best_dist = 0;
+        for (int64_t c = 0; c < n; ++c) {
+            if (taken[c]) continue;
+            int64_t dist = 0;
+            for (int64_t w = 0; w < words; ++w) {
+                uint32_t x = qcode[w] ^ codes[c * words + w];
+                while (x) { dist += x & 1u; x >>= 1; }
+            }
+            if (best < 0 || dist < best_dist) { best = c; best_dist = dist; }
+        }
+        taken[best] = 1;
+    }
+    int64_t m = 0;
+    for (int64_t c = 0; c < n; ++c) if (taken[c]) out[m++] = c;
+    *n_out = m;
+    free(taken);
+    return 0;
+}

@@ -333,3 +333,79 @@ def decode_paged(q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, rows
         O[b] = o[0, :, 0, :]
         LSE[b] = ls[0, :, 0]
     return O, LSE
+
+
+# ---- L3 recall: sign-random-projection codes and top-R selection (a reading; the paper names no hash) ----------------
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def srp_code(x, proj) -> np.ndarray:
+    """Code of one vector x[d] under proj[bits, d]: bit j = [proj[j] . x >= 0], the dot product taken as one fp32 fmaf
+    chain over the columns.  Returns uint32[bits // 32], bit j in word j // 32 at position j % 32."""
+    x, proj = _f32(x), _f32(proj)
+    bits, d = proj.shape
+    code = np.zeros(bits // 32, dtype=np.uint32)
+    rc = _load().orc_srp_code(x.ctypes.data_as(ctypes.c_void_p), proj.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(d),
+                              ctypes.c_int64(bits), code.ctypes.data_as(ctypes.c_void_p))
+    assert rc == 0
+    return code
+
+
+def sum_rows_f32(x) -> np.ndarray:
+    """Column sums of x[n, d] accumulated row by row in fp32."""
+    x = _f32(x)
+    s = np.zeros(x.shape[1], dtype=np.float32)
+    _load().orc_sum_rows_f32(x.ctypes.data_as(ctypes.c_void_p), ctypes.c_int64(x.shape[0]), ctypes.c_int64(x.shape[1]),
+                             s.ctypes.data_as(ctypes.c_void_p))
+    return s
+
+
+def l3_index(pool_k, proj) -> np.ndarray:
+    """Codes of every (page, KV head) of a key pool [P, H_kv, page_rows, d]: the code of the sum of the page's keys.
+    Returns uint32 [P, H_kv, bits // 32]."""
+    pool_k = _f32(pool_k)
+    P, H_kv = pool_k.shape[:2]
+    out = np.zeros((P, H_kv, proj.shape[0] // 32), dtype=np.uint32)
+    for pg in range(P):
+        for h in range(H_kv):
+            out[pg, h] = srp_code(sum_rows_f32(pool_k[pg, h]), proj)
+    return out
+
+
+def l3_select(qcode, codes, R: int):
+    """Indices (ascending) of the min(R, n) rows of codes[n, words] nearest to qcode in Hamming distance, ties to the
+    lower index."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint32)
+    qcode = np.ascontiguousarray(qcode, dtype=np.uint32)
+    n, words = codes.shape
+    out = np.zeros(max(R, 1), dtype=np.int64)
+    n_out = ctypes.c_int64(0)
+    rc = _load().orc_l3_select(qcode.ctypes.data_as(ctypes.c_void_p), codes.ctypes.data_as(ctypes.c_void_p),
+                               ctypes.c_int64(n), ctypes.c_int64(words), ctypes.c_int64(R),
+                               out.ctypes.data_as(ctypes.c_void_p), ctypes.byref(n_out))
+    assert rc == 0
+    return out[:n_out.value].copy()
+
+
+def l3_retrieve(q, proj, codes, bank, bank_len, R: int, H_kv: int):
+    """Retrieve of Alg. 2 step 4 under the reading above.  q [B, H, d]; codes [P, H_kv, words] from l3_index;
+    bank [B, n] pool pages of each sequence's long-term chunks in time order, bank_len [B] how many are in use.
+    For every (sequence, KV head): the query is the fp32 sum of the query heads sharing the KV head (head order), its
+    code is compared with the codes of the sequence's bank and the pool pages of the R nearest chunks are returned
+    in bank order.  Returns (table int32 [B, H_kv, R], zero-padded; n_sel int32 [B])."""
+    q = _f32(q)
+    B, H, d = q.shape
+    G = H // H_kv
+    table = np.zeros((B, H_kv, R), dtype=np.int32)
+    n_sel = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        n = int(bank_len[b])
+        pages = np.asarray(bank[b][:n], dtype=np.int64)
+        for h in range(H_kv):
+            qc = srp_code(sum_rows_f32(q[b, h * G:(h + 1) * G]), proj)
+            pos = l3_select(qc, codes[pages, h], R) if n else np.zeros(0, dtype=np.int64)
+            table[b, h, :len(pos)] = pages[pos]
+            n_sel[b] = len(pos)
+    return table, n_sel
