@@ -159,13 +159,15 @@ mka_status mka_decode(const mka_shape* shape, const void* q, const mka_level L[3
 /* One memory level kept in PAGES (the paged KV layout the paper's inference setup uses for contexts beyond 32K):
  * pools k, v hold fixed-size pages; element (page, kv head, row, :) sits at page*stride_page + head*stride_h +
  * row*stride_n (ELEMENTS, d contiguous).  Logical row r of sequence b is row r % page_rows of pool page
- * page_table[b*table_stride + r / page_rows].  n may be 0 (then the pointers may be NULL). */
+ * page_table[b*table_stride + h*table_head_stride + r / page_rows].  n may be 0 (then the pointers may be NULL). */
 typedef struct mka_paged_level {
     const void *k, *v;          /* device, bf16 */
     const int32_t* page_table;  /* device [B, table_stride]; entries of pages that hold no valid row are never read */
     const int32_t* rows;        /* device [B]: valid rows of every sequence (clamped to [0, n]), or NULL = n for all */
     int64_t n;                  /* upper bound of the sequences' rows (host); table_stride * page_rows >= n */
     int64_t table_stride;
+    int64_t table_head_stride;  /* 0 = one table per sequence; else KV head h of sequence b uses the table at
+                                   b*table_stride + h*table_head_stride (per-head recall lists of mka_l3_retrieve) */
     int32_t page_rows;          /* rows per page: a power of two */
     int64_t stride_page, stride_h, stride_n;
 } mka_paged_level;
@@ -183,6 +185,37 @@ typedef struct mka_paged_level {
 size_t mka_decode_paged_workspace_bytes(const mka_shape* shape, int32_t H_kv, const int64_t n_level[3]);
 mka_status mka_decode_paged(const mka_shape* shape, int32_t H_kv, const void* q, const mka_paged_level L[3],
                             const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * L3 recall (Alg. 2 step 4 "L3 <- Retrieve(Q_h)"; the method section's vectorized hashing with chunk-based recall; the
+ * passkey table recalls R = 8 chunks per query).  The paper does not define the hash; this library's reading: a chunk
+ * is one page of the long-term key pool, its signature a sign-random-projection code of the SUM of its keys
+ * (bit j = [proj[j] . sum >= 0]); the query of a KV head is the sum of the query heads that share it; the R chunks of
+ * the sequence's bank whose codes agree with the query's code in the most bits are recalled, ties to the earlier
+ * chunk, and listed in bank (time) order.  Code bits are decided in fp32: sums run row by row (head by head for the
+ * query), a projection is one fmaf chain over the columns 0..d-1.
+ *
+ * mka_l3_index: codes of every (page, KV head) of a key pool.
+ *   k_pool   bf16 pool, element (page, head, row, :) at page*stride_page + head*stride_h + row*stride_n; all
+ *            page_rows rows of a page are summed (unused rows of a partly filled page must be zero)
+ *   proj     [bits, d] f32, bits in {32, 64, 128, 256}; d in {64, 128}
+ *   codes    [n_pages, H_kv, bits/32] uint32 out: bit j of a code is bit j%32 of word j/32
+ * mka_l3_retrieve: per (sequence, KV head) the page table of the recalled chunks.
+ *   q        [B, H, d] bf16;  codes from mka_l3_index with the same proj
+ *   bank     int32 [B, bank_stride]: pool pages of each sequence's long-term chunks in time order; bank_len int32 [B]
+ *            how many are in use (clamped to [0, max_bank]); max_bank (host) <= bank_stride, at most 32768
+ *   R        chunks to recall, 1..64
+ *   table    int32 [B, H_kv, R] out: recalled pool pages in bank order, unused slots 0
+ *   n_sel    int32 [B] out or NULL: min(R, bank_len[b]);  rows int32 [B] out or NULL: n_sel * page_rows
+ * The outputs plug into mka_paged_level (page_table = table, table_stride = H_kv*R, table_head_stride = R, rows).
+ */
+mka_status mka_l3_index(const void* k_pool, int64_t n_pages, int32_t H_kv, int32_t page_rows, int32_t d,
+                        int64_t stride_page, int64_t stride_h, int64_t stride_n, const float* proj, int32_t bits,
+                        uint32_t* codes, void* stream);
+mka_status mka_l3_retrieve(const void* q, int32_t B, int32_t H, int32_t H_kv, int32_t d, const float* proj,
+                           int32_t bits, const uint32_t* codes, const int32_t* bank, const int32_t* bank_len,
+                           int64_t bank_stride, int32_t max_bank, int32_t R, int32_t page_rows, int32_t* table,
+                           int32_t* n_sel, int32_t* rows, void* stream);
 
 /*
  * Backward of mka_fwd in MKA_MODE_FAST (derived from Eq. 5; the paper prints no backward).  With

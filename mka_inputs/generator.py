@@ -236,3 +236,49 @@ def make_paged(cfg: PagedConfig, device="cpu"):
     g = approx_normal(cfg.seed, 27, 0, cfg.B * 3, 1.0, device, torch.float32).view(cfg.B, 3).abs() + 0.05
     return {"q": q, "pools_k": pk, "pools_v": pv, "tables": [t.to(device) for t in tables],
             "rows": [r.to(device) for r in paged_rows(cfg)], "gate_raw": g}
+
+
+# ---- L3 recall: a long-term bank of chunks (pages) per sequence ----------------------------------------------------------
+
+@dataclass(frozen=True)
+class RecallConfig:
+    """B sequences whose long-term memory holds `bank` chunks (pages of page_rows rows) each; H query heads on H_kv KV
+    heads of width d; `bits`-bit codes; R chunks recalled per (sequence, KV head).  `len_frac[b % len]` scales how much
+    of the bank sequence b uses."""
+    name: str
+    seed: int
+    B: int
+    H: int
+    H_kv: int
+    d: int
+    bank: int
+    page_rows: int
+    bits: int
+    R: int
+    len_frac: Tuple[float, ...] = (1.0,)
+
+
+RECALL_CONFIGS: Dict[str, RecallConfig] = {
+    # 128K tokens of long-term memory per sequence in 16-row chunks, top-8 recall (the passkey table's R)
+    "r3": RecallConfig("r3", 9, 4, 28, 4, 128, 8192, 16, 64, 8),
+    "r3p": RecallConfig("r3p", 9, 1, 28, 4, 128, 8192, 16, 64, 8),
+    "r1": RecallConfig("r1", 10, 3, 12, 4, 64, 37, 8, 32, 8, len_frac=(1.0, 0.1, 0.0)),
+}
+
+
+def make_recall(cfg: RecallConfig, device="cpu"):
+    """q [B, H, d] bf16; pools_k / pools_v [B * bank + 1, H_kv, page_rows, d] bf16; proj [bits, d] f32; bank int32
+    [B, bank]: the pool pages of every sequence's chunks, dealt from a seeded shuffle; bank_len int32 [B]."""
+    P = cfg.B * cfg.bank + 1
+    shape = (P, cfg.H_kv, cfg.page_rows, cfg.d)
+    cnt = shape[0] * shape[1] * shape[2] * shape[3]
+    out = {"q": approx_normal(cfg.seed, 30, 0, cfg.B * cfg.H * cfg.d, 1.0, device, torch.bfloat16).view(cfg.B, cfg.H, cfg.d),
+           "pool_k": approx_normal(cfg.seed, 31, 0, cnt, 1.0, device, torch.bfloat16).view(shape),
+           "pool_v": approx_normal(cfg.seed, 32, 0, cnt, 1.0, device, torch.bfloat16).view(shape),
+           "proj": approx_normal(cfg.seed, 33, 0, cfg.bits * cfg.d, 1.0, device, torch.float32).view(cfg.bits, cfg.d)}
+    gen = torch.Generator().manual_seed(cfg.seed * 1000 + 7)
+    order = torch.randperm(P, generator=gen).to(torch.int32)
+    out["bank"] = order[:cfg.B * cfg.bank].view(cfg.B, cfg.bank).contiguous().to(device)
+    out["bank_len"] = torch.tensor([int(cfg.bank * cfg.len_frac[b % len(cfg.len_frac)]) for b in range(cfg.B)],
+                                   dtype=torch.int32, device=device)
+    return out

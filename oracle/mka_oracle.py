@@ -306,7 +306,8 @@ def decode_paged(q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, rows
     """Single-token decode of Eq. 5 over paged levels with grouped-query sharing of the KV heads.
 
     q [B, H, d]; for level l: pools_k[l], pools_v[l] [P_l, H_kv, page_rows, d] (or None for an absent level),
-    tables[l] [B, pages] page table, rows[l] [B] valid rows of every sequence; gate [B, 3].
+    tables[l] [B, pages] page table (or [B, H_kv, pages]: one per KV head, as L3 recall produces), rows[l] [B] valid
+    rows of every sequence; gate [B, 3].
     Query head h reads KV head h // (H / H_kv): consecutive query heads share one KV head.
     Every sequence is gathered into dense levels and handed to the dense decode (all gathered rows visible).
     Returns O [B, H, d], LSE [B, H]."""
@@ -324,8 +325,15 @@ def decode_paged(q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, rows
                 continue
             H_kv = np.asarray(pools_k[l]).shape[1]
             assert H % H_kv == 0
-            kd = gather_pages(_f64(pools_k[l]), tables[l][b], int(rows[l][b]), page_rows)
-            vd = gather_pages(_f64(pools_v[l]), tables[l][b], int(rows[l][b]), page_rows)
+            tab = np.asarray(tables[l][b])
+            if tab.ndim == 2:                                    # one recall list per KV head: gather head by head
+                kd = np.concatenate([gather_pages(_f64(pools_k[l])[:, h:h + 1], tab[h], int(rows[l][b]), page_rows)
+                                     for h in range(H_kv)], axis=0)
+                vd = np.concatenate([gather_pages(_f64(pools_v[l])[:, h:h + 1], tab[h], int(rows[l][b]), page_rows)
+                                     for h in range(H_kv)], axis=0)
+            else:
+                kd = gather_pages(_f64(pools_k[l]), tab, int(rows[l][b]), page_rows)
+                vd = gather_pages(_f64(pools_v[l]), tab, int(rows[l][b]), page_rows)
             share = np.arange(H) // (H // H_kv)                  # KV head of every query head
             Ks.append(kd[share][None])
             Vs.append(vd[share][None])

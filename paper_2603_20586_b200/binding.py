@@ -26,7 +26,7 @@ TILE = 128
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
            "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_l2_summary_workspace_bytes", "mka_l2_summary_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes",
-           "mka_decode_paged", "mka_decode_paged_workspace_bytes"]
+           "mka_decode_paged", "mka_decode_paged_workspace_bytes", "mka_l3_index", "mka_l3_retrieve"]
 
 
 class MkaError(RuntimeError):
@@ -48,7 +48,7 @@ class mka_level_grad(ctypes.Structure):
 class mka_paged_level(ctypes.Structure):
     _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("page_table", ctypes.c_void_p),
                 ("rows", ctypes.c_void_p), ("n", ctypes.c_int64), ("table_stride", ctypes.c_int64),
-                ("page_rows", ctypes.c_int32), ("stride_page", ctypes.c_int64), ("stride_h", ctypes.c_int64),
+                ("table_head_stride", ctypes.c_int64), ("page_rows", ctypes.c_int32), ("stride_page", ctypes.c_int64), ("stride_h", ctypes.c_int64),
                 ("stride_n", ctypes.c_int64)]
 
 
@@ -98,6 +98,8 @@ def _load() -> ctypes.CDLL:
     lib.mka_decode_paged_workspace_bytes.argtypes = [ctypes.POINTER(mka_shape), i32, ctypes.POINTER(ctypes.c_int64)]
     lib.mka_decode_paged.argtypes = [ctypes.POINTER(mka_shape), i32, vp, ctypes.POINTER(mka_paged_level), vp, vp, vp, vp,
                                      ctypes.c_size_t, vp]
+    lib.mka_l3_index.argtypes = [vp, i64, i32, i32, i32, i64, i64, i64, vp, i32, vp, vp]
+    lib.mka_l3_retrieve.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.mka_l2_summary_kernel_kind.argtypes = [i32, i64, i32, i32, ctypes.c_size_t]
     lib.mka_l2_summary.argtypes = [vp, i32, i64, i32, i32, i32, ctypes.c_float, vp, i64, vp, vp, ctypes.c_size_t, vp]
     lib.mka_bwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level), vp]
@@ -227,16 +229,17 @@ def _paged_levels(pools_k, pools_v, tables, rows, n):
     for l in range(3):
         k, v = pools_k[l], pools_v[l]
         if k is None or n[l] == 0:
-            arr[l] = mka_paged_level(None, None, None, None, 0, 0, 1, 0, 0, 0)
+            arr[l] = mka_paged_level(None, None, None, None, 0, 0, 0, 1, 0, 0, 0)
             continue
         # pools [pages, H_kv, page_rows, d]; any strides with d contiguous
         assert k.dim() == 4 and k.stride(3) == 1 and v.stride() == k.stride() and v.shape == k.shape
         tab = tables[l]
-        assert tab.dtype == torch.int32 and tab.dim() == 2 and tab.stride(1) == 1
+        # [B, pages]: one table per sequence; [B, H_kv, pages]: one per (sequence, KV head)
+        assert tab.dtype == torch.int32 and tab.dim() in (2, 3) and tab.stride(-1) == 1
         r = None if rows is None else rows[l]
         assert r is None or (r.dtype == torch.int32 and r.is_contiguous())
         arr[l] = mka_paged_level(k.data_ptr(), v.data_ptr(), tab.data_ptr(), _ptr(r), int(n[l]), tab.stride(0),
-                                 k.shape[2], k.stride(0), k.stride(1), k.stride(2))
+                                 tab.stride(1) if tab.dim() == 3 else 0, k.shape[2], k.stride(0), k.stride(1), k.stride(2))
     return arr
 
 
@@ -258,6 +261,37 @@ def mka_decode_paged(shape: mka_shape, H_kv: int, q, pools_k, pools_v, tables, n
     _check(lib.mka_decode_paged(ctypes.byref(shape), H_kv, _ptr(q), _paged_levels(pools_k, pools_v, tables, rows, n),
                                 _ptr(gate), _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream)), "mka_decode_paged")
     return O, LSE
+
+
+def mka_l3_index(pool_k, proj, codes=None, stream=None):
+    """Sign-random-projection codes of every (page, KV head) of a key pool [pages, H_kv, page_rows, d] under
+    proj [bits, d] f32; returns int32 [pages, H_kv, bits // 32] holding the code words' bit patterns."""
+    assert pool_k.dim() == 4 and pool_k.stride(3) == 1 and proj.dtype == torch.float32 and proj.is_contiguous()
+    P, H_kv, pr, d = pool_k.shape
+    bits = proj.shape[0]
+    if codes is None:
+        codes = torch.empty(P, H_kv, bits // 32, dtype=torch.int32, device=pool_k.device)
+    _check(lib.mka_l3_index(_ptr(pool_k), P, H_kv, pr, d, pool_k.stride(0), pool_k.stride(1), pool_k.stride(2), _ptr(proj),
+                            bits, _ptr(codes), _stream(stream)), "mka_l3_index")
+    return codes
+
+
+def mka_l3_retrieve(q, H_kv: int, proj, codes, bank, bank_len, R: int, page_rows: int, table=None, n_sel=None, rows=None,
+                    stream=None):
+    """Recall lists of every (sequence, KV head): returns (table int32 [B, H_kv, R], n_sel int32 [B], rows int32 [B])."""
+    assert q.is_contiguous() and bank.dtype == torch.int32 and bank.dim() == 2 and bank.stride(1) == 1
+    assert bank_len.dtype == torch.int32 and bank_len.is_contiguous() and codes.is_contiguous()
+    B, H, d = q.shape
+    if table is None:
+        table = torch.empty(B, H_kv, R, dtype=torch.int32, device=q.device)
+    if n_sel is None:
+        n_sel = torch.empty(B, dtype=torch.int32, device=q.device)
+    if rows is None:
+        rows = torch.empty(B, dtype=torch.int32, device=q.device)
+    _check(lib.mka_l3_retrieve(_ptr(q), B, H, H_kv, d, _ptr(proj), proj.shape[0], _ptr(codes), _ptr(bank), _ptr(bank_len),
+                               bank.stride(0), bank.shape[1], R, page_rows, _ptr(table), _ptr(n_sel), _ptr(rows),
+                               _stream(stream)), "mka_l3_retrieve")
+    return table, n_sel, rows
 
 
 def mka_decode_static(shape: mka_shape, q, K, V, gate, O, LSE=None, stream=None):

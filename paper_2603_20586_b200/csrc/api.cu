@@ -247,14 +247,18 @@ mka_status mka_decode_paged(const mka_shape* s, int32_t H_kv, const void* q, con
         if (!L[l].k || !L[l].v || !L[l].page_table) return MKA_ERR_ARG;
         const int pr = L[l].page_rows;
         if (pr <= 0 || (pr & (pr - 1)) != 0) return MKA_ERR_SHAPE;
-        if (L[l].table_stride * pr < L[l].n) return MKA_ERR_SHAPE;
+        {   // the table of one (sequence, head) must hold the pages of n rows
+            const int64_t width = L[l].table_head_stride > 0 ? L[l].table_head_stride : L[l].table_stride;
+            if (width * pr < L[l].n) return MKA_ERR_SHAPE;
+        }
         if (L[l].stride_n < s->d || L[l].stride_page < 0 || L[l].stride_h < 0) return MKA_ERR_SHAPE;
         if (!aligned16(L[l].k) || !aligned16(L[l].v)) return MKA_ERR_ALIGN;
         if (L[l].stride_n % 8 || L[l].stride_page % 8 || L[l].stride_h % 8) return MKA_ERR_ALIGN;
         int shift = 0;
         while ((1 << shift) < pr) ++shift;
         p.L[l].k = L[l].k; p.L[l].v = L[l].v; p.L[l].table = L[l].page_table; p.L[l].rows = L[l].rows;
-        p.L[l].n = L[l].n; p.L[l].table_stride = L[l].table_stride;
+        if (L[l].table_head_stride < 0) return MKA_ERR_SHAPE;
+        p.L[l].n = L[l].n; p.L[l].table_stride = L[l].table_stride; p.L[l].table_head_stride = L[l].table_head_stride;
         p.L[l].sp = L[l].stride_page; p.L[l].sh = L[l].stride_h; p.L[l].sn = L[l].stride_n;
         p.L[l].page_shift = shift;
     }
@@ -281,6 +285,37 @@ mka_status mka_decode_paged(const mka_shape* s, int32_t H_kv, const void* q, con
     cudaError_t e = launch_decode_paged(p, cs);
     if (e == cudaSuccess) e = launch_decode_combine(c, cs);
     if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
+mka_status mka_l3_index(const void* k_pool, int64_t n_pages, int32_t H_kv, int32_t page_rows, int32_t d,
+                        int64_t stride_page, int64_t stride_h, int64_t stride_n, const float* proj, int32_t bits,
+                        uint32_t* codes, void* stream) {
+    if (n_pages < 0 || H_kv < 0 || page_rows <= 0) return MKA_ERR_SHAPE;
+    if (d != 64 && d != 128) return MKA_ERR_SHAPE;
+    if (bits != 32 && bits != 64 && bits != 128 && bits != 256) return MKA_ERR_SHAPE;
+    if (n_pages == 0 || H_kv == 0) return MKA_OK;
+    if (!k_pool || !proj || !codes) return MKA_ERR_ARG;
+    if (stride_n < d || stride_page < 0 || stride_h < 0) return MKA_ERR_SHAPE;
+    if (!aligned16(k_pool) || stride_n % 8 || stride_page % 8 || stride_h % 8) return MKA_ERR_ALIGN;
+    cudaError_t e = launch_l3_index(k_pool, n_pages, H_kv, page_rows, d, stride_page, stride_h, stride_n, proj, bits, codes,
+                                    static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
+mka_status mka_l3_retrieve(const void* q, int32_t B, int32_t H, int32_t H_kv, int32_t d, const float* proj,
+                           int32_t bits, const uint32_t* codes, const int32_t* bank, const int32_t* bank_len,
+                           int64_t bank_stride, int32_t max_bank, int32_t R, int32_t page_rows, int32_t* table,
+                           int32_t* n_sel, int32_t* rows, void* stream) {
+    if (B < 0 || H < 0 || H_kv <= 0 || (H > 0 && H % H_kv != 0)) return MKA_ERR_SHAPE;
+    if (d != 64 && d != 128) return MKA_ERR_SHAPE;
+    if (bits != 32 && bits != 64 && bits != 128 && bits != 256) return MKA_ERR_SHAPE;
+    if (R < 1 || R > 64 || page_rows <= 0) return MKA_ERR_SHAPE;
+    if (max_bank < 0 || max_bank > 32768 || bank_stride < max_bank) return MKA_ERR_SHAPE;
+    if (B == 0 || H == 0) return MKA_OK;
+    if (!q || !proj || !codes || !bank || !bank_len || !table) return MKA_ERR_ARG;
+    cudaError_t e = launch_l3_retrieve(q, B, H, H_kv, d, proj, bits, codes, bank, bank_len, bank_stride, max_bank, R,
+                                       page_rows, table, n_sel, rows, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
 }
 

@@ -106,7 +106,7 @@ struct PagedLevelDev {
     const void* v;
     const int* table;    // [B, table_stride]
     const int* rows;     // [B] or null
-    long long n, table_stride, sp, sh, sn;
+    long long n, table_stride, table_head_stride, sp, sh, sn;
     int page_shift;      // log2(page_rows)
 };
 struct DecodePagedParams {
@@ -121,6 +121,11 @@ struct DecodePagedParams {
     float* partial;      // [B*H, total_chunks, d+2]
 };
 cudaError_t launch_decode_paged(const DecodePagedParams& p, cudaStream_t st);
+cudaError_t launch_l3_index(const void* k, long long n_pages, int H_kv, int page_rows, int d, long long sp, long long sh,
+                            long long sn, const float* proj, int bits, unsigned int* codes, cudaStream_t st);
+cudaError_t launch_l3_retrieve(const void* q, int B, int H, int H_kv, int d, const float* proj, int bits,
+                               const unsigned int* codes, const int* bank, const int* bank_len, long long bank_stride,
+                               int max_bank, int R, int page_rows, int* table, int* n_sel, int* rows, cudaStream_t st);
 
 struct BwdParams {
     const void *Q, *O, *dO;

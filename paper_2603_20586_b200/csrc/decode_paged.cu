@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_paged_kernel(const DecodeP
     __shared__ int s_pages[kMaxChunkRows];
     const long long page0 = r_begin >> shift;
     {
-        const int* table = L.table + (long long)b * L.table_stride + page0;
+        const int* table = L.table + (long long)b * L.table_stride + (long long)kvh * L.table_head_stride + page0;
         const int n_pages = (int)(((r_end - 1) >> shift) - page0) + 1;
         for (int i = tid; i < n_pages; i += kThreads) s_pages[i] = table[i];
     }

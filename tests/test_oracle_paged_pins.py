@@ -89,3 +89,19 @@ def test_result_does_not_depend_on_where_the_pages_live(orc):
         tab2.append(perm[tab[l]].astype(np.int32))
     O2, L2 = orc.decode_paged(q, pk2, pv2, tab2, rows, pr, g)
     assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+
+
+def test_per_head_tables_that_agree_equal_the_shared_table(orc):
+    rng = np.random.default_rng(8)
+    B, H, H_kv, d, pr = 2, 4, 2, 8, 4
+    rows = [np.array([6, 3]), np.array([9, 12]), np.array([8, 8])]
+    q, pk, pv, tab, g = _case(rng, B, H, H_kv, d, pr, rows)
+    O1, L1 = orc.decode_paged(q, pk, pv, tab, rows, pr, g)
+    per_head = [np.repeat(t[:, None, :], H_kv, axis=1) for t in tab]
+    O2, L2 = orc.decode_paged(q, pk, pv, per_head, rows, pr, g)
+    assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+    # and a table that differs between the heads moves only the heads of that KV head
+    per_head[1][0, 1] = per_head[1][0, 1][::-1].copy()
+    O3, _ = orc.decode_paged(q, pk, pv, per_head, rows, pr, g)
+    assert np.array_equal(O3[0, :2], O1[0, :2]) and not np.array_equal(O3[0, 2:], O1[0, 2:])
+    assert np.array_equal(O3[1], O1[1])
