@@ -31,7 +31,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from mka_inputs import CONFIGS, PAGED_CONFIGS, make_paged, make_tensor  # noqa: E402
+from mka_inputs import CONFIGS, PAGED_CONFIGS, RECALL_CONFIGS, make_paged, make_recall, make_tensor  # noqa: E402
 
 DATASHEET = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
@@ -67,7 +67,9 @@ def ncu_traffic(key, cfg):
     ent = NCU_TRAFFIC.get(key)
     if ent is None:
         return None
-    if key.startswith("decode_paged"):
+    if key.startswith("l3_index"):
+        units = cfg.B                                                      # one sequence's bank
+    elif key.startswith("decode_paged"):
         units = cfg.B * cfg.H_kv                                           # one KV head of one sequence
     else:
         units = cfg.B if key.startswith("l2_summary") else cfg.B * cfg.H     # the summary's unit is a whole sequence
@@ -138,6 +140,9 @@ class Leg:
         self.mka, self.name, self.dev = mka, name, device
         if name in PAGED_CONFIGS:
             self._init_paged(PAGED_CONFIGS[name], device, seed_shift)
+            return
+        if name in RECALL_CONFIGS:
+            self._init_recall(RECALL_CONFIGS[name], device, seed_shift)
             return
         cfg = CONFIGS[name]
         if seed_shift:
@@ -212,8 +217,52 @@ class Leg:
         self.launches_per_step = 2
         self.ev = []
 
+    def _init_recall(self, cfg, device, seed_shift):
+        """L3 recall: index the long-term key pool, recall R chunks per (sequence, KV head), decode over them."""
+        import dataclasses
+        mka = self.mka
+        if seed_shift:
+            cfg = dataclasses.replace(cfg, seed=cfg.seed + 1000 * seed_shift)
+        self.cfg, self.kind = cfg, "recall"
+        P = make_recall(cfg, device)
+        self.t = {"q": P["q"], "pool_k": P["pool_k"], "pool_v": P["pool_v"]}
+        self.proj, self.bank, self.bank_len = P["proj"], P["bank"], P["bank_len"]
+        self.codes = torch.empty(P["pool_k"].shape[0], cfg.H_kv, cfg.bits // 32, dtype=torch.int32, device=device)
+        self.table = torch.empty(cfg.B, cfg.H_kv, cfg.R, dtype=torch.int32, device=device)
+        self.n_sel = torch.empty(cfg.B, dtype=torch.int32, device=device)
+        self.rows3 = torch.empty(cfg.B, dtype=torch.int32, device=device)
+        self.gate_d = torch.tensor([[0.0, 0.0, 1.0]] * cfg.B, device=device)
+        self.shape = mka.make_shape(cfg.B, cfg.H, 1, cfg.d, 32)
+        self.n3 = cfg.R * cfg.page_rows
+        self.Od = torch.empty_like(P["q"])
+        self.LSEd = torch.empty(cfg.B, cfg.H, device=device)
+        self.ws = torch.zeros(mka.mka_decode_paged_workspace_bytes(self.shape, cfg.H_kv, [0, 0, self.n3]), dtype=torch.uint8,
+                              device=device)
+        k = P["pool_k"]
+        # the index kernel reads every key of the pool once and writes bits/8 bytes per (page, KV head)
+        self.work = {"index_bytes": float(k.numel() * 2 + self.codes.numel() * 4)}
+        self.launches_per_step = 4              # index, retrieve, decode partial, decode combine
+        self.ev = []
+
     def step(self, record=False):
         mka, t = self.mka, self.t
+        if self.kind == "recall":
+            cfg = self.cfg
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
+            if record:
+                e[0].record(); e[1].record()
+            mka.mka_l3_index(t["pool_k"], self.proj, codes=self.codes)
+            if record:
+                e[2].record()
+            mka.mka_l3_retrieve(t["q"], cfg.H_kv, self.proj, self.codes, self.bank, self.bank_len, cfg.R, cfg.page_rows,
+                                table=self.table, n_sel=self.n_sel, rows=self.rows3)
+            mka.mka_decode_paged(self.shape, cfg.H_kv, t["q"], [None, None, t["pool_k"]], [None, None, t["pool_v"]],
+                                 [None, None, self.table], [0, 0, self.n3], self.gate_d, rows=[None, None, self.rows3],
+                                 O=self.Od, LSE=self.LSEd, ws=self.ws)
+            if record:
+                e[3].record()
+                self.ev.append(e)
+            return
         if self.kind == "paged":
             e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
             if record:
@@ -256,7 +305,7 @@ class Leg:
             self.ev.append(e)
 
     def result_tensor(self):
-        if self.kind == "paged":
+        if self.kind in ("paged", "recall"):
             return self.Od
         if self.kind == "summary":
             return self.M2
@@ -296,7 +345,15 @@ def timed_steps(leg, steps, warmup, dist=None):
 
 def leg_report(leg, ms_per_step, n_gpus, peaks):
     cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
-    if leg.kind == "paged":
+    if leg.kind == "recall":
+        # main = the index kernel; "bwd" holds the recall-list kernel plus the decode over the recalled chunks
+        achieved = w["index_bytes"] / (k["main"] * 1e-3) / 1e9
+        roof = {"kernel": "l3_index_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
+                "peak_source": peaks["source"], "traffic": ncu_traffic("l3_index_kernel@r3", cfg) if leg.name[:2] == "r3" else None}
+        value = n_gpus * w["index_bytes"] / (ms_per_step * 1e-3) / 1e9
+        unit, metric = "GB/s", "l3_recall_hbm_gbs"
+    elif leg.kind == "paged":
         achieved = w["decode_bytes"] / (k["main"] * 1e-3) / 1e9
         roof = {"kernel": "decode_paged_kernel+decode_combine_kernel", "bound": "hbm", "achieved": achieved,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
@@ -409,9 +466,28 @@ def oracle_sample_paged(name):
             "sample": f"one sequence of the configuration's {PAGED_CONFIGS[name].B}: all {cfg.H} heads, all {int(sum(int(r.sum()) for r in rows))} cached rows"}
 
 
+def oracle_sample_recall(name):
+    """The oracle index + recall lists on one sequence of the configuration."""
+    import dataclasses
+    from oracle import mka_oracle as orc
+    full = RECALL_CONFIGS[name]
+    cfg = dataclasses.replace(full, B=1)
+    P = make_recall(cfg, "cpu")
+    pool, proj = P["pool_k"].float().numpy(), P["proj"].numpy()
+    t0 = time.perf_counter()
+    codes = orc.l3_index(pool, proj)
+    orc.l3_retrieve(P["q"].float().numpy(), proj, codes, P["bank"].numpy(), P["bank_len"].numpy(), cfg.R, cfg.H_kv)
+    dt = time.perf_counter() - t0
+    bytes_ = float(pool.size * 2 + codes.size * 4)
+    return {"value": bytes_ / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dt,
+            "sample": f"index and recall lists of {cfg.bank} of sequence 0's {full.bank} chunks (one thread)"}
+
+
 def oracle_sample(name, budget_rows=None):
     if name in PAGED_CONFIGS:
         return oracle_sample_paged(name)
+    if name in RECALL_CONFIGS:
+        return oracle_sample_recall(name)
     """Times the CPU oracle, as it stands, on a bounded seeded sample of workload `name`."""
     from oracle import mka_oracle as orc
     orc.build()
@@ -502,8 +578,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "s3", "g4", "c3p", "c4p", "c5p", "f3p", "s3p", "g4p"])
-    ap.add_argument("--legs", default="c4,c5,c2,f3,s3,g4", help="other configurations measured after the primary one ('' = none)")
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "s3", "g4", "r3", "c3p", "c4p", "c5p", "f3p", "s3p", "g4p", "r3p"])
+    ap.add_argument("--legs", default="c4,c5,c2,f3,s3,g4,r3", help="other configurations measured after the primary one ('' = none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -512,11 +588,13 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     wk = args.workload[:2]
-    paged = args.workload in PAGED_CONFIGS
-    cfg = PAGED_CONFIGS[args.workload] if paged else CONFIGS[args.workload]
+    paged = args.workload in PAGED_CONFIGS or args.workload in RECALL_CONFIGS
+    cfg = PAGED_CONFIGS.get(args.workload) or RECALL_CONFIGS.get(args.workload) or CONFIGS[args.workload]
     metric_name = {"c4": "decode_hbm_gbs", "c5": "fwd_bwd_tflops", "f3": "route_fuse_hbm_gbs", "s3": "l2_summary_hbm_gbs",
-                   "g4": "decode_paged_hbm_gbs"}.get(wk, "prefill_fwd_tflops")
-    describe = (f"{args.workload}: B={cfg.B} H={cfg.H} H_kv={cfg.H_kv} d={cfg.d} N={list(cfg.N)} page_rows={cfg.page_rows} seed={cfg.seed}"
+                   "g4": "decode_paged_hbm_gbs", "r3": "l3_recall_hbm_gbs"}.get(wk, "prefill_fwd_tflops")
+    describe = (f"{args.workload}: B={cfg.B} H={cfg.H} H_kv={cfg.H_kv} d={cfg.d} bank={cfg.bank} chunks x {cfg.page_rows} rows, {cfg.bits}-bit codes, R={cfg.R} seed={cfg.seed}"
+                if args.workload in RECALL_CONFIGS else
+                f"{args.workload}: B={cfg.B} H={cfg.H} H_kv={cfg.H_kv} d={cfg.d} N={list(cfg.N)} page_rows={cfg.page_rows} seed={cfg.seed}"
                 if paged else
                 f"{args.workload}: B={cfg.B} H={cfg.H} d={cfg.d} D={cfg.D} T={cfg.T} W={cfg.W} N={list(cfg.N)} seed={cfg.seed}")
     base = {"metric": f"FastMKA {metric_name} (algorithmic, visible pairs only)", "n_gpus": args.gpus, "steps": args.steps,
@@ -569,7 +647,9 @@ def main():
     if not args.no_e2e:
         e_ms, h2d, d2h = e2e_run(leg, max(2, min(args.steps, 5)), 1)
         w = leg.work
-        if wk in ("c4", "g4"):
+        if wk == "r3":
+            ev = world * w["index_bytes"] / (e_ms * 1e-3) / 1e9
+        elif wk in ("c4", "g4"):
             ev = world * w["decode_bytes"] / (e_ms * 1e-3) / 1e9
         elif wk == "f3":
             ev = world * w["fuse_bytes"] / (e_ms * 1e-3) / 1e9

@@ -12,9 +12,9 @@
 namespace mka {
 namespace {
 
-constexpr int kIdxThreads = 256;
-constexpr int kIdxLanes = 16;                         // threads per (page, head): 8 columns each for d = 128
-constexpr int kIdxPairs = kIdxThreads / kIdxLanes;    // (page, head) pairs per batch of a CTA
+constexpr int kIdxThreads = 128;
+constexpr int kIdxPairs = 32;                         // (page, head) pairs per batch of a CTA: one per lane in the projections
+constexpr int kIdxBitsPerWarp = 16;                   // code bits one warp works out per pass
 
 struct L3IndexParams {
     const __nv_bfloat16* k;
@@ -24,74 +24,102 @@ struct L3IndexParams {
     int H_kv, page_rows, d, bits;
 };
 
-// dynamic shared memory: projT [d][bits] floats, then s [kIdxPairs][d] floats
-__global__ void __launch_bounds__(kIdxThreads) l3_index_kernel(const L3IndexParams p) {
+// Dynamic shared memory: projT [d][bits + 4] floats (16 consecutive bits of one column are one broadcast read), then
+// s [kIdxPairs][d + 1] floats (the key sums; the odd pitch keeps the lanes of a warp on different banks).
+// A batch = 32 (page, head) pairs.  Loading: 16 threads cover one 256-byte row, a thread sums its eight columns row by
+// row.  Projections: lane = pair, warp = 16 bits; column i costs one read of s, four broadcast reads of projT and 16
+// fmaf, so the arithmetic, not shared memory, is what the projections wait for.
+template <int DH>
+__global__ void __launch_bounds__(kIdxThreads, 4) l3_index_kernel(const L3IndexParams p) {
     extern __shared__ __align__(16) float sm[];
+    const int ppitch = p.bits + 4;                             // floats between columns of projT (keeps the fill off one bank)
     float* projT = sm;
-    float* s = sm + (size_t)p.d * p.bits;
-    const int tid = threadIdx.x;
-    for (int e = tid; e < p.d * p.bits; e += kIdxThreads) {
-        const int j = e / p.d, i = e % p.d;
-        projT[i * p.bits + j] = p.proj[e];
+    float* s = sm + (size_t)DH * ppitch;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int pitch = DH + 1;
+    for (int e = tid; e < DH * p.bits; e += kIdxThreads) {     // e = j * d + i: coalesced reads of proj
+        const int j = e / DH, i = e % DH;
+        projT[i * ppitch + j] = p.proj[e];
     }
-    const int lane16 = tid % kIdxLanes, slot = tid / kIdxLanes;
-    const int vecs = p.d / 8;                                  // 16-byte pieces of a row: 16 (d = 128) or 8 (d = 64)
+    constexpr int vecs = DH / 8;                               // 16-byte pieces of a row: 16 (d = 128) or 8 (d = 64)
+    constexpr int items = kIdxPairs * vecs;                    // (pair, piece) items of a batch
+    constexpr int kPerThread = items / kIdxThreads;            // 4 or 2: taken two at a time, 16 loads in flight
     const long long pairs = p.n_pages * p.H_kv;
     const int words = p.bits / 32;
+    unsigned short* codes16 = reinterpret_cast<unsigned short*>(p.codes);
     for (long long base = (long long)blockIdx.x * kIdxPairs; base < pairs; base += (long long)gridDim.x * kIdxPairs) {
         __syncthreads();                                       // projT is there; the previous batch is done with s
-        const long long pair = base + slot;
-        // ---- sums of the page's keys, row by row, eight columns per thread
-        if (pair < pairs && lane16 < vecs) {
-            const long long pg = pair / p.H_kv, h = pair % p.H_kv;
-            const __nv_bfloat16* src = p.k + pg * p.sp + h * p.sh + lane16 * 8;
-            float acc[8];
+        // ---- sums of the pages' keys, row by row
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        for (int k0 = 0; k0 < kPerThread; k0 += 2) {
+            float acc[2][8];
+            const __nv_bfloat16* src[2];
+            bool live[2];
+            int slot[2], piece[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int it = tid + (k0 + q) * kIdxThreads;
+                slot[q] = it / vecs; piece[q] = it % vecs;
+                const long long pair = base + slot[q];
+                live[q] = pair < pairs;
+                const long long pc = live[q] ? pair : 0;
+                src[q] = p.k + (pc / p.H_kv) * p.sp + (pc % p.H_kv) * p.sh + piece[q] * 8;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[q][i] = 0.f;
+            }
             for (int r0 = 0; r0 < p.page_rows; r0 += 8) {
-                uint4 u[8];
+                uint4 u[2][8];
 #pragma unroll
-                for (int r = 0; r < 8; ++r)
-                    if (r0 + r < p.page_rows) u[r] = *reinterpret_cast<const uint4*>(src + (long long)(r0 + r) * p.sn);
+                for (int q = 0; q < 2; ++q)
 #pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    if (r0 + r < p.page_rows) {
-                        const uint32_t w[4] = {u[r].x, u[r].y, u[r].z, u[r].w};
+                    for (int r = 0; r < 8; ++r)
+                        u[q][r] = (live[q] && r0 + r < p.page_rows)
+                                      ? __ldg(reinterpret_cast<const uint4*>(src[q] + (long long)(r0 + r) * p.sn))
+                                      : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            acc[2 * i] = acc[2 * i] + __uint_as_float(w[i] << 16);
-                            acc[2 * i + 1] = acc[2 * i + 1] + __uint_as_float(w[i] & 0xffff0000u);
+                for (int q = 0; q < 2; ++q)
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        if (r0 + r < p.page_rows) {                // rows past the page add nothing, not even +0
+                            const uint32_t w[4] = {u[q][r].x, u[q][r].y, u[q][r].z, u[q][r].w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                acc[q][2 * i] = acc[q][2 * i] + __uint_as_float(w[i] << 16);
+                                acc[q][2 * i + 1] = acc[q][2 * i + 1] + __uint_as_float(w[i] & 0xffff0000u);
+                            }
                         }
                     }
-                }
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) s[slot * p.d + lane16 * 8 + i] = acc[i];
+            for (int q = 0; q < 2; ++q)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) s[slot[q] * pitch + piece[q] * 8 + i] = acc[q][i];
         }
         __syncthreads();
-        // ---- projections: thread = (pair, four consecutive bits of a 64-bit group); one fmaf chain per bit
-        {
-            const bool valid = pair < pairs;                   // every lane runs the shuffles below
-            const float* sv = s + slot * p.d;
-            for (int g0 = 0; g0 < p.bits; g0 += 64) {
-                const int j0 = g0 + 4 * lane16;
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-                if (valid && j0 < p.bits) {
-                    for (int i = 0; i < p.d; ++i) {
-                        const float4 pr = *reinterpret_cast<const float4*>(projT + i * p.bits + j0);
-                        const float x = sv[i];
-                        a0 = fmaf(pr.x, x, a0); a1 = fmaf(pr.y, x, a1); a2 = fmaf(pr.z, x, a2); a3 = fmaf(pr.w, x, a3);
-                    }
+        // ---- projections: one fmaf chain per (pair, bit) over the columns 0..d-1
+        const long long pair = base + lane;
+        const float* sv = s + lane * pitch;
+        for (int j0 = warp * kIdxBitsPerWarp; j0 < p.bits; j0 += (kIdxThreads / 32) * kIdxBitsPerWarp) {
+            float a[kIdxBitsPerWarp];
+#pragma unroll
+            for (int j = 0; j < kIdxBitsPerWarp; ++j) a[j] = 0.f;
+            const float* pj = projT + j0;
+            for (int i = 0; i < DH; ++i) {
+                const float x = sv[i];
+#pragma unroll
+                for (int v = 0; v < kIdxBitsPerWarp / 4; ++v) {
+                    const float4 pr = *reinterpret_cast<const float4*>(pj + (size_t)i * ppitch + 4 * v);
+                    a[4 * v] = fmaf(pr.x, x, a[4 * v]);
+                    a[4 * v + 1] = fmaf(pr.y, x, a[4 * v + 1]);
+                    a[4 * v + 2] = fmaf(pr.z, x, a[4 * v + 2]);
+                    a[4 * v + 3] = fmaf(pr.w, x, a[4 * v + 3]);
                 }
-                unsigned nib = (a0 >= 0.f ? 1u : 0u) | (a1 >= 0.f ? 2u : 0u) | (a2 >= 0.f ? 4u : 0u) | (a3 >= 0.f ? 8u : 0u);
-                if (j0 >= p.bits) nib = 0u;
-                unsigned word = nib << (4 * (lane16 & 7));     // lanes 0-7 fill the group's first word, 8-15 the second
-                word |= __shfl_xor_sync(0xffffffffu, word, 1);
-                word |= __shfl_xor_sync(0xffffffffu, word, 2);
-                word |= __shfl_xor_sync(0xffffffffu, word, 4);
-                const int w = g0 / 32 + (lane16 >> 3);
-                if (valid && (lane16 & 7) == 0 && w < words) p.codes[pair * words + w] = word;
             }
+            unsigned half = 0u;
+#pragma unroll
+            for (int j = 0; j < kIdxBitsPerWarp; ++j) half |= (a[j] >= 0.f ? 1u : 0u) << j;
+            // bits j0..j0+15 are one 16-bit half of word j0 / 32 (low half first)
+            if (pair < pairs) codes16[(pair * words) * 2 + j0 / 16] = (unsigned short)half;
         }
     }
 }
@@ -199,15 +227,18 @@ cudaError_t launch_l3_index(const void* k, long long n_pages, int H_kv, int page
     L3IndexParams p;
     p.k = static_cast<const __nv_bfloat16*>(k); p.proj = proj; p.codes = codes;
     p.n_pages = n_pages; p.sp = sp; p.sh = sh; p.sn = sn; p.H_kv = H_kv; p.page_rows = page_rows; p.d = d; p.bits = bits;
-    const size_t smem = ((size_t)d * bits + (size_t)kIdxPairs * d) * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(l3_index_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const size_t smem = ((size_t)d * (bits + 4) + (size_t)kIdxPairs * (d + 1)) * sizeof(float);
+    auto kern = d == 128 ? l3_index_kernel<128> : l3_index_kernel<64>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const long long batches = (n_pages * H_kv + kIdxPairs - 1) / kIdxPairs;
-    const long long resident = 148LL * (smem > 100 * 1024 ? 1 : (smem > 48 * 1024 ? 2 : 4));
-    // a few batches per CTA amortise the transposed projection in shared memory
-    long long grid = batches < resident * 4 ? (batches + 3) / 4 : resident;
-    if (grid < 1) grid = 1;
-    l3_index_kernel<<<(unsigned)grid, kIdxThreads, smem, st>>>(p);
+    const long long per_sm = smem > 110 * 1024 ? 1 : (smem > 72 * 1024 ? 2 : (smem > 54 * 1024 ? 3 : 4));
+    const long long resident = 148LL * per_sm;
+    // persistent CTAs: every CTA transposes the projection into shared memory once and then walks its batches
+    // (the grid is shrunk so that all CTAs get the same number of batches)
+    const long long per_cta = (batches + resident - 1) / resident;
+    const long long grid = (batches + per_cta - 1) / per_cta;
+    kern<<<(unsigned)grid, kIdxThreads, smem, st>>>(p);
     return cudaGetLastError();
 }
 

@@ -172,3 +172,35 @@ def test_c5_training_forward_backward(mka, orc):
         for l in range(3):
             _bf16_ok(np64(g["dK"][l][b, h]), r["dK"][l][0, 0], f"dK{l}[{b},{h}]")
             _bf16_ok(np64(g["dV"][l][b, h]), r["dV"][l][0, 0], f"dV{l}[{b},{h}]")
+
+
+def test_g4_paged_grouped_query_decode_full_size(mka, orc):
+    """Workload g4 as bench.py launches it; the oracle evaluates sequence 0 (all 28 heads, all 143360 cached rows)."""
+    from mka_inputs import PAGED_CONFIGS, make_paged
+    cfg = PAGED_CONFIGS["g4"]
+    P = make_paged(cfg, "cuda")
+    gate = (P["gate_raw"] / P["gate_raw"].sum(1, keepdim=True)).contiguous()
+    shape = mka.make_shape(cfg.B, cfg.H, 1, cfg.d, 32)
+    O, LSE = mka.mka_decode_paged(shape, cfg.H_kv, P["q"], P["pools_k"], P["pools_v"], P["tables"], list(cfg.N), gate,
+                                  rows=P["rows"])
+    i64 = lambda t: t.cpu().numpy().astype(np.int64)
+    Or, Lr = orc.decode_paged(np64(P["q"][:1]), [np64(k) for k in P["pools_k"]], [np64(v) for v in P["pools_v"]],
+                              [i64(t[:1]) for t in P["tables"]], [i64(r[:1]) for r in P["rows"]], cfg.page_rows, np64(gate[:1]))
+    _bf16_ok(np64(O[:1]), Or, "g4 O")
+    assert np.abs(np64(LSE[:1]) - Lr).max() <= 2e-3
+    assert torch.isfinite(O.float()).all() and torch.isfinite(LSE).all()
+
+
+def test_r3_recall_full_size_is_bit_exact(mka, orc):
+    """Workload r3: codes of the whole pool and the recall lists of every (sequence, KV head) against the oracle."""
+    from mka_inputs import RECALL_CONFIGS, make_recall
+    cfg = RECALL_CONFIGS["r3"]
+    P = make_recall(cfg, "cuda")
+    codes = mka.mka_l3_index(P["pool_k"], P["proj"])
+    proj = P["proj"].cpu().numpy()
+    want = orc.l3_index(P["pool_k"].float().cpu().numpy(), proj)
+    assert np.array_equal(codes.cpu().numpy().view(np.uint32), want)
+    table, n_sel, rows = mka.mka_l3_retrieve(P["q"], cfg.H_kv, P["proj"], codes, P["bank"], P["bank_len"], cfg.R, cfg.page_rows)
+    t_ref, n_ref = orc.l3_retrieve(P["q"].float().cpu().numpy(), proj, want, P["bank"].cpu().numpy(), P["bank_len"].cpu().numpy(),
+                                   cfg.R, cfg.H_kv)
+    assert np.array_equal(table.cpu().numpy(), t_ref) and np.array_equal(n_sel.cpu().numpy(), n_ref)
