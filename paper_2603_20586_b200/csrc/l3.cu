@@ -170,11 +170,36 @@ __global__ void __launch_bounds__(kRetThreads) l3_retrieve_kernel(const L3Retrie
     int n = p.bank_len[b];
     n = n < 0 ? 0 : (n > p.max_bank ? p.max_bank : n);
     const int* bank = p.bank + (long long)b * p.bank_stride;
-    for (int c = tid; c < n; c += kRetThreads) {
-        const unsigned int* code = p.codes + ((long long)bank[c] * p.H_kv + kvh) * words;
-        int dist = 0;
-        for (int w = 0; w < words; ++w) dist += __popc(code[w] ^ qcode[w]);
-        score[c] = (unsigned short)(p.bits - dist);            // agreement: 0..bits (<= 256)
+    // eight chunks per thread at a time: the page numbers first, then all their code words, so that the two dependent
+    // gathers cost two round trips per eight chunks and not two per chunk
+    for (int c0 = tid; c0 < n; c0 += 8 * kRetThreads) {
+        int page[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int c = c0 + u * kRetThreads;
+            page[u] = c < n ? bank[c] : 0;
+        }
+        if (words == 2) {                                      // 64-bit codes: one 8-byte load per chunk
+            uint2 w[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                w[u] = __ldg(reinterpret_cast<const uint2*>(p.codes + ((long long)page[u] * p.H_kv + kvh) * 2));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int c = c0 + u * kRetThreads;
+                if (c < n) score[c] = (unsigned short)(p.bits - __popc(w[u].x ^ qcode[0]) - __popc(w[u].y ^ qcode[1]));
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int c = c0 + u * kRetThreads;
+                if (c >= n) continue;
+                const unsigned int* code = p.codes + ((long long)page[u] * p.H_kv + kvh) * words;
+                int dist = 0;
+                for (int w = 0; w < words; ++w) dist += __popc(__ldg(code + w) ^ qcode[w]);
+                score[c] = (unsigned short)(p.bits - dist);    // agreement: 0..bits (<= 256)
+            }
+        }
     }
     __syncthreads();
     const int k = p.R < n ? p.R : n;
