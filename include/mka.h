@@ -274,14 +274,15 @@ typedef enum { MKA_SUMMARY_MEAN = 0, MKA_SUMMARY_EMA = 1 } mka_summary;
  *           are single-pass and give the same results up to fp32 summation order.  NULL = no scratch, no status word.
  * fp32 arithmetic, one rounding to the storage type.  Counts are converted to f32 (exact up to 2^24 tokens).
  */
+mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_t dtype, int32_t kind, float beta,
+                          float* state, int64_t n_prev, void* M2, void* ws, size_t ws_bytes, void* stream);
 /* Scratch bytes that let mka_l2_summary use its segmented form: 512 + 8 bytes per segment and column (about 1.6 % of
  * a bf16 input).  The call clears the scratch on its stream, so its contents on entry do not matter.  Host only. */
 size_t mka_l2_summary_workspace_bytes(int32_t B, int64_t T, int32_t D, int32_t dtype);
 /* 1 when mka_l2_summary would run the segmented form for this input with ws_bytes of scratch (T >= 512, enough
  * scratch, and for fp32 fewer than 96 strips of 128 bytes over all sequences), else 0 (the strip form).  Host only. */
 int32_t mka_l2_summary_kernel_kind(int32_t B, int64_t T, int32_t D, int32_t dtype, size_t ws_bytes);
-mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_t dtype, int32_t kind, float beta,
-                          float* state, int64_t n_prev, void* M2, void* ws, size_t ws_bytes, void* stream);
+
 
 /*
  * Decode for callers that cannot provide scratch memory (the paper has no counterpart; this entry

@@ -24,6 +24,9 @@
  *                       separately; used only to test Theorem 1 and block-wise == full.
  *   orc_bwd_head        gradients of <dO, O> for O of Eq. 5; derived by differentiating
  *                       Eq. 5 (the paper prints no backward).
+ *   orc_sum_rows_f32, orc_srp_code, orc_l3_select   the L3 recall of Alg. 2 step 4 under the
+ *                       sign-random-projection reading described above them (fp32 by definition,
+ *                       because floating point decides the code bits).
  *
  * All arrays are row-major doubles.  One call handles one (batch, head) problem:
  *   Q[T][d], K_l[n_l][d], V_l[n_l][d], gate[T][3].

@@ -2,7 +2,8 @@
 
 Nothing in the product package may import this module; it exists so that the
 tests, the smoke check and the benchmark's cpu-baseline leg can evaluate the
-paper's definitions (Eq. 5, Alg. 1, the router, the derived backward) in fp64.
+paper's definitions (Eq. 5, Alg. 1, the router, the derived backward) in fp64, and the steps around
+them (route-fusion, session summary, paged grouped-query decode, L3 recall).
 
 The wrappers only marshal arrays: they loop over (batch, head), hand one head
 problem at a time to the C routines, and sum the per-head router-logit
