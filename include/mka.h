@@ -179,7 +179,8 @@ typedef struct mka_paged_level {
  * (head h reads KV head h / (H / H_kv)); H must be a multiple of H_kv with at most 16 query heads per KV head.
  * Every cached row is read once per KV head.  A level whose gate is exactly 0 for a sequence is not read.
  *   q [B, H, d] bf16;  gate [B, 3] f32;  O [B, H, d] bf16;  LSE [B, H] f32 or NULL
- *   ws: mka_decode_paged_workspace_bytes(shape, H_kv, n_level) bytes, n_level[l] = L[l].n
+ *   ws: mka_decode_paged_workspace_bytes(shape, H_kv, n_level) bytes, n_level[l] = L[l].n.  The levels are split into
+ *       chunks of a multiple of 128 rows (at most 8192), chosen so that the grid makes few rounds of the resident CTAs
  * d must be 64 or 128; pools 16-byte aligned with strides that are multiples of 8 elements.
  */
 size_t mka_decode_paged_workspace_bytes(const mka_shape* shape, int32_t H_kv, const int64_t n_level[3]);

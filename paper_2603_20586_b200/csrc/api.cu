@@ -222,10 +222,41 @@ mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], c
     return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
 }
 
+// Split table of the paged decode.  Its CTAs are few and long-lived (two per SM, one KV head's rows each), so what
+// counts is how many rounds of resident CTAs the grid makes and what every CTA pays to start (page-table slice, first
+// tiles: about as long as streaming 256 rows).  Pick the chunk length, a multiple of 128 rows, with the least
+// rounds x (rows + 256).
+static mka_status paged_plan(const int64_t n_level[3], int32_t B, int32_t H_kv, mka_decode_plan_t* plan) {
+    if (!n_level || !plan) return MKA_ERR_ARG;
+    if (B < 0 || H_kv < 0) return MKA_ERR_SHAPE;
+    for (int l = 0; l < 3; ++l) if (n_level[l] < 0) return MKA_ERR_SHAPE;
+    const int64_t resident = 148 * 2;
+    const int64_t groups = (int64_t)B * H_kv > 0 ? (int64_t)B * H_kv : 1;
+    int64_t best_rows = 128, best_cost = -1;
+    for (int64_t rows = 128; rows <= 8192; rows += 128) {
+        int64_t chunks = 0, longest = 0;
+        for (int l = 0; l < 3; ++l) {
+            chunks += (n_level[l] + rows - 1) / rows;
+            const int64_t len = n_level[l] < rows ? n_level[l] : rows;
+            longest = len > longest ? len : longest;
+        }
+        const int64_t rounds = (chunks * groups + resident - 1) / resident;
+        const int64_t cost = rounds * (longest + 256);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_rows = rows; }
+    }
+    plan->chunk_rows = best_rows;
+    plan->total_chunks = 0;
+    for (int l = 0; l < 3; ++l) {
+        plan->n_chunks[l] = (n_level[l] + best_rows - 1) / best_rows;
+        plan->total_chunks += plan->n_chunks[l];
+    }
+    return MKA_OK;
+}
+
 size_t mka_decode_paged_workspace_bytes(const mka_shape* s, int32_t H_kv, const int64_t n_level[3]) {
     if (!s || !n_level || H_kv <= 0 || s->B < 0 || s->H < 0 || s->d <= 0) return 0;
     mka_decode_plan_t plan;
-    if (mka_decode_plan(n_level, s->B, H_kv, s->d, &plan) != MKA_OK) return 0;
+    if (paged_plan(n_level, s->B, H_kv, &plan) != MKA_OK) return 0;
     return kWsHeader + round_up((size_t)s->B * s->H * plan.total_chunks * (s->d + 2) * sizeof(float), 256);
 }
 
@@ -268,7 +299,7 @@ mka_status mka_decode_paged(const mka_shape* s, int32_t H_kv, const void* q, con
     const size_t need = mka_decode_paged_workspace_bytes(s, H_kv, n_level);
     if (!ws || ws_bytes < need) return MKA_ERR_WORKSPACE;
     mka_decode_plan_t plan;
-    mka_decode_plan(n_level, s->B, H_kv, s->d, &plan);
+    paged_plan(n_level, s->B, H_kv, &plan);
     if ((long long)s->B * s->H * plan.total_chunks > 0x7fffffffLL) return MKA_ERR_SHAPE;
     p.q = q; p.gate = gate;
     p.B = s->B; p.H = s->H; p.H_kv = H_kv; p.d = s->d; p.scale = resolve_scale(s);

@@ -21,7 +21,7 @@ namespace {
 constexpr int kThreads = 128;
 constexpr int kTileRows = 64;
 constexpr int kStages = 3;
-constexpr int kMaxChunkRows = 1024;                  // the split table never makes longer chunks
+constexpr int kSliceCap = 1024;                      // page-table entries of a chunk kept in shared memory
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -100,13 +100,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_paged_kernel(const DecodeP
     const int shift = L.page_shift;
     const long long page_mask = ((long long)1 << shift) - 1;
     // this chunk's slice of the page table, fetched once: at most one entry per row of the chunk
-    __shared__ int s_pages[kMaxChunkRows];
+    __shared__ int s_pages[kSliceCap];
     const long long page0 = r_begin >> shift;
-    {
-        const int* table = L.table + (long long)b * L.table_stride + (long long)kvh * L.table_head_stride + page0;
-        const int n_pages = (int)(((r_end - 1) >> shift) - page0) + 1;
-        for (int i = tid; i < n_pages; i += kThreads) s_pages[i] = table[i];
-    }
+    const int* table = L.table + (long long)b * L.table_stride + (long long)kvh * L.table_head_stride + page0;
+    const long long n_pages = ((r_end - 1) >> shift) - page0 + 1;
+    const bool sliced = n_pages <= kSliceCap;              // (tiny pages in a long chunk: look the table up in place)
+    if (sliced)
+        for (int i = tid; i < (int)n_pages; i += kThreads) s_pages[i] = table[i];
     __syncthreads();
     const __nv_bfloat16* Kbase = static_cast<const __nv_bfloat16*>(L.k) + (long long)kvh * L.sh;
     const __nv_bfloat16* Vbase = static_cast<const __nv_bfloat16*>(L.v) + (long long)kvh * L.sh;
@@ -120,7 +120,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_paged_kernel(const DecodeP
             const int rr = pass * kRowsPerPass + prow;
             long long r = base + rr;
             if (r >= r_end) r = r_end - 1;                  // a tail row re-reads the last valid row (masked later)
-            const long long off = (long long)s_pages[(r >> shift) - page0] * L.sp + (r & page_mask) * L.sn + piece * 8;
+            const long long pi = (r >> shift) - page0;
+            const long long off = (long long)(sliced ? s_pages[pi] : table[pi]) * L.sp + (r & page_mask) * L.sn + piece * 8;
             cp_async16(smem_addr(sK + rr * kPitch + piece * 16), Kbase + off);
             cp_async16(smem_addr(sV + rr * kPitch + piece * 16), Vbase + off);
         }
@@ -249,7 +250,6 @@ template <int DH>
 cudaError_t launch_t(const DecodePagedParams& p, cudaStream_t st) {
     const long long ctas = (long long)p.B * p.H_kv * p.total_chunks;
     if (ctas == 0) return cudaSuccess;
-    if (p.chunk_rows > kMaxChunkRows) return cudaErrorInvalidValue;
     const size_t smem = (size_t)kStages * 2 * kTileRows * (DH * 2 + 16);
     cudaError_t e = cudaFuncSetAttribute(decode_paged_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
