@@ -1,6 +1,6 @@
 // Causal L2 session summary, segmented form: the scan of summary.cu for inputs that offer too few column strips to
-// fill the GPU (one long sequence).  The sequence is cut into segments of kSegRows rows; a tile is one segment of one
-// 128-byte column strip (32 KB, read from DRAM once into shared memory).  Persistent CTAs take tiles from a ticket
+// fill the GPU (one long sequence).  The sequence is cut into segments of 256 or 512 rows; a tile is one segment of one
+// 128- or 64-byte column strip (32 KB, read from DRAM once into shared memory).  Persistent CTAs take tiles from a ticket
 // counter and, per tile,
 //   1. total their rows with a zero incoming state: the segment acts on the carried state as the affine pair
 //      (a, b) = (beta^rows, total) [prefix mean: (1, sum)]; publish b and raise the segment's flag to AGGREGATE;
@@ -20,8 +20,9 @@ namespace {
 
 constexpr int kSegThreads = 128;
 constexpr int kSegCtasPerSm = 6;                     // one 32 KB tile each
-constexpr int kSegBytesPerRow = 128;                 // strip width: one full line per row
-constexpr int kSegRows = 256;                        // rows per segment: a 32 KB tile
+constexpr int kSegTileBytes = 32768;                 // a tile: WB bytes of every row of a segment of 32768 / WB rows
+constexpr int kSegMinRows = 256;                     // the shortest segment (WB = 128): sizes the scratch
+constexpr int kSegBoxRows = 256;                     // rows of one TMA box; a tile is one or two of them
 constexpr unsigned kFlagAggregate = 1u, kFlagInclusive = 2u;
 
 struct SegParams {
@@ -84,17 +85,22 @@ __device__ __forceinline__ void st_rec2(unsigned long long* p, unsigned flag, fl
 __device__ __forceinline__ unsigned rec_flag(unsigned long long r) { return (unsigned)(r >> 32); }
 __device__ __forceinline__ float rec_val(unsigned long long r) { return __uint_as_float((unsigned)r); }
 
-template <typename T, bool kEma>
+// WB = strip width in bytes (128 or 64).  The fewer strips an input offers, the narrower they are made: segments
+// of one strip that are in flight at the same time wait for each other in the look-back, and with N strips about
+// 888 / N of them are (measured on [1, 32768, D] inputs: 64 strips 0.76 of the copy bandwidth, 128 strips 0.82,
+// 256 strips 0.94).  A narrower strip has longer segments, so a tile stays 32 KB and a thread's share 32 rows x 8 bytes.
+template <typename T, bool kEma, int WB>
 __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_kernel(const __grid_constant__ CUtensorMap map, const SegParams p) {
     using P2 = typename Pair2<T>::type;
-    constexpr int kNC = kSegBytesPerRow / (int)sizeof(T);     // columns of the strip: 64 (bf16) or 32 (f32)
+    constexpr int kSegRows = kSegTileBytes / WB;               // rows per segment: 256 or 512
+    constexpr int kNC = WB / (int)sizeof(T);                   // columns of the strip
     constexpr int kNP = kNC / 2;                               // column pairs: what one lane of the look-back warp carries
     constexpr int CW = Oct<T>::kCols;                          // columns of one thread in the scans: 8 bytes of a row
-    constexpr int kNL = kNC / CW;                              // threads across a row: 16
-    constexpr int G = kSegThreads / kNL;                       // row groups: 8
+    constexpr int kNL = kNC / CW;                              // threads across a row: 16 or 8
+    constexpr int G = kSegThreads / kNL;                       // row groups: 8 or 16
     constexpr int RG = kSegRows / G;                           // rows scanned by one thread: 32
     using V8 = typename Oct<T>::type;
-    constexpr uint32_t kTileBytes = kSegRows * kSegBytesPerRow;
+    constexpr uint32_t kTileBytes = kSegTileBytes;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     __shared__ float part[G][kNC];
@@ -148,7 +154,9 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
         unsigned nxt = 0;
         if (tid == 0) {
             mbar_expect_tx(&full, kTileBytes);
-            tma_load_3d(smem, &map, col0, row0, b, &full);
+#pragma unroll
+            for (int bx = 0; bx < kSegRows / kSegBoxRows; ++bx)
+                tma_load_3d(smem + (size_t)bx * kSegBoxRows * WB, &map, col0, row0 + bx * kSegBoxRows, b, &full);
             pending_s = it & 1;
             nxt = atomicAdd(p.ticket, 1u);                     // the next place; needed only at the end of this tile
         }
@@ -333,18 +341,30 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
     }
 }
 
+template <typename T, bool kEma, int WB>
+cudaError_t launch_w(const void* X, SegParams p, cudaStream_t st) {
+    constexpr int kNC = WB / (int)sizeof(T);
+    constexpr int kRows = kSegTileBytes / WB;
+    p.S = (int)((p.T + kRows - 1) / kRows);
+    p.strips = (p.D + kNC - 1) / kNC;
+    const long long tiles = (long long)p.S * p.B * p.strips;
+    if (tiles > 0x7fffffffLL) return cudaErrorNotSupported;
+    CUtensorMap map;
+    if (!make_strip_map(&map, X, sizeof(T) == 2, p.D, p.T, p.B, kNC, kSegBoxRows)) return cudaErrorNotSupported;
+    const size_t smem = (size_t)kSegTileBytes + 128;
+    cudaError_t e = cudaFuncSetAttribute(l2_summary_seg_kernel<T, kEma, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const long long resident = (long long)kSegCtasPerSm * 148;
+    l2_summary_seg_kernel<T, kEma, WB><<<(unsigned)(tiles < resident ? tiles : resident), kSegThreads, smem, st>>>(map, p);
+    return cudaGetLastError();
+}
+
+// Strip width: 128 bytes when all sequences together offer about 200 strips, else 64.
 template <typename T, bool kEma>
 cudaError_t launch_k(const void* X, const SegParams& p, cudaStream_t st) {
-    constexpr int kNC = kSegBytesPerRow / (int)sizeof(T);
-    CUtensorMap map;
-    if (!make_strip_map(&map, X, sizeof(T) == 2, p.D, p.T, p.B, kNC, kSegRows)) return cudaErrorNotSupported;
-    const size_t smem = (size_t)kSegRows * kSegBytesPerRow + 128;
-    cudaError_t e = cudaFuncSetAttribute(l2_summary_seg_kernel<T, kEma>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    const long long tiles = (long long)p.S * p.B * p.strips;
-    const long long resident = (long long)kSegCtasPerSm * 148;                                 // three CTAs fit one SM
-    l2_summary_seg_kernel<T, kEma><<<(unsigned)(tiles < resident ? tiles : resident), kSegThreads, smem, st>>>(map, p);
-    return cudaGetLastError();
+    const long long strips128 = (long long)p.B * ((p.D * (long long)sizeof(T) + 127) / 128);
+    if (strips128 >= 192) return launch_w<T, kEma, 128>(X, p, st);
+    return launch_w<T, kEma, 64>(X, p, st);          // 32-byte strips were measured too: they lose more in DRAM efficiency than they gain
 }
 
 }  // namespace
@@ -352,7 +372,7 @@ cudaError_t launch_k(const void* X, const SegParams& p, cudaStream_t st) {
 // Scratch of the segmented form: the ticket counter and one 8-byte record per segment and column.
 size_t l2_summary_seg_workspace(int B, long long T, int D, int dtype) {
     (void)dtype;
-    const long long S = (T + kSegRows - 1) / kSegRows;
+    const long long S = (T + kSegMinRows - 1) / kSegMinRows;      // the widest strips have the most segments
     return 256 + (size_t)B * S * D * sizeof(unsigned long long);
 }
 
@@ -361,10 +381,7 @@ cudaError_t launch_l2_summary_seg(const void* X, void* M2, float* state, int use
     if (B == 0 || T == 0 || D == 0) return cudaSuccess;
     if (!tensor_map_encoder_available()) return cudaErrorNotSupported;
     SegParams p;
-    p.S = (int)((T + kSegRows - 1) / kSegRows);
-    const int nc = kSegBytesPerRow / (dtype == MKA_BF16 ? 2 : 4);
-    p.strips = (D + nc - 1) / nc;
-    if ((long long)p.S * B * p.strips > 0x7fffffffLL) return cudaErrorNotSupported;
+    p.S = 0; p.strips = 0;                                        // set per strip width at launch
     p.ticket = static_cast<unsigned int*>(scratch);
     p.rec = reinterpret_cast<unsigned long long*>(static_cast<char*>(scratch) + 256);
     p.M2 = M2; p.state = state; p.T = T; p.n_prev = n_prev; p.B = B; p.D = D; p.kind = kind; p.beta = beta;
