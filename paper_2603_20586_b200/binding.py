@@ -56,7 +56,7 @@ class mka_shape(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("D", ctypes.c_int32), ("window", ctypes.c_int32), ("q_offset", ctypes.c_int32),
                 ("scale", ctypes.c_float), ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32),
-                ("flags", ctypes.c_uint32)]
+                ("flags", ctypes.c_uint32), ("kv_heads", ctypes.c_int32)]
 
 
 class mka_decode_plan_t(ctypes.Structure):
@@ -144,8 +144,9 @@ def _n_level(n) -> ctypes.Array:
     return (ctypes.c_int64 * 3)(*[int(x) for x in n])
 
 
-def make_shape(B, H, T, d, D=0, window=1, q_offset=0, scale=0.0, dtype=MKA_BF16, mode=MKA_MODE_FAST, flags=0) -> mka_shape:
-    return mka_shape(B, H, T, d, D, window, q_offset, scale, dtype, mode, flags)
+def make_shape(B, H, T, d, D=0, window=1, q_offset=0, scale=0.0, dtype=MKA_BF16, mode=MKA_MODE_FAST, flags=0,
+               kv_heads=0) -> mka_shape:
+    return mka_shape(B, H, T, d, D, window, q_offset, scale, dtype, mode, flags, kv_heads)
 
 
 def _levels(K: Sequence[Optional[torch.Tensor]], V: Sequence[Optional[torch.Tensor]]):

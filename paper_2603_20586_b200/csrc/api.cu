@@ -21,6 +21,7 @@ mka_status check_shape(const mka_shape* s, bool decode) {
     if (!decode && s->window < 1) return MKA_ERR_SHAPE;
     if (!decode && s->q_offset < 0) return MKA_ERR_SHAPE;
     if (decode && s->T != 1) return MKA_ERR_SHAPE;
+    if (s->kv_heads < 0 || (s->kv_heads > 0 && s->H % s->kv_heads != 0)) return MKA_ERR_SHAPE;
     return MKA_OK;
 }
 
@@ -39,6 +40,7 @@ mka_status check_levels(const mka_shape* s, const mka_level L[3]) {
     return MKA_OK;
 }
 
+int kv_group_of(const mka_shape* s) { return s->kv_heads > 0 ? s->H / s->kv_heads : 1; }
 float resolve_scale(const mka_shape* s) { return s->scale > 0.f ? s->scale : 1.0f / sqrtf((float)s->d); }
 
 void fill_levels(LevelDev out[3], const mka_level L[3]) {
@@ -169,7 +171,7 @@ mka_status mka_fwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     fill_levels(p.L, L);
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
     p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s);
-    p.mode = s->mode; p.decode = 0;
+    p.mode = s->mode; p.decode = 0; p.kv_group = kv_group_of(s);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
     cudaError_t e;
@@ -186,7 +188,7 @@ int32_t mka_fwd_kernel_kind(const mka_shape* s, const mka_level L[3]) {
     FwdParams p;
     memset(&p, 0, sizeof(p));
     fill_levels(p.L, L);
-    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.mode = s->mode;
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.mode = s->mode; p.kv_group = kv_group_of(s);
     return (!(s->flags & MKA_FLAG_FORCE_SIMT) && s->mode == MKA_MODE_FAST && fwd_tc_eligible(p, s->dtype)) ? 1 : 0;
 }
 
@@ -210,7 +212,7 @@ mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], c
     memset(&p, 0, sizeof(p));
     p.q = q; p.O = O; p.LSE = LSE; p.gate = gate;
     fill_levels(p.L, L);
-    p.B = s->B; p.H = s->H; p.d = s->d; p.scale = resolve_scale(s);
+    p.B = s->B; p.H = s->H; p.d = s->d; p.scale = resolve_scale(s); p.kv_group = kv_group_of(s);
     p.chunk_rows = plan.chunk_rows;
     for (int l = 0; l < 3; ++l) p.n_chunks[l] = plan.n_chunks[l];
     p.total_chunks = plan.total_chunks;
@@ -357,6 +359,7 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     mka_status st = check_shape(s, false);
     if (st != MKA_OK) return st;
     if (s->mode != MKA_MODE_FAST) return MKA_ERR_UNSUPPORTED;
+    if (kv_group_of(s) != 1) return MKA_ERR_UNSUPPORTED;      // gradients of shared KV heads: not built
     if ((st = check_levels(s, L)) != MKA_OK) return st;
     if (!dL) return MKA_ERR_ARG;
     for (int l = 0; l < 3; ++l) {

@@ -42,6 +42,7 @@ struct FwdParams {
     float scale;        // tau
     int mode;
     int decode;         // every row visible
+    int kv_group;       // query heads per KV head (>= 1): head h reads KV head h / kv_group
 };
 
 template <typename T> struct Elem;
@@ -92,6 +93,7 @@ struct DecodeParams {
     const float* gate;   // [B,3]
     LevelDev L[3];
     int B, H, d;
+    int kv_group;        // query heads per KV head (>= 1)
     float scale;
     long long chunk_rows;
     long long n_chunks[3];

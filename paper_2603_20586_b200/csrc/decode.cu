@@ -53,8 +53,8 @@ __global__ void __launch_bounds__(kWarps * 32, 2) decode_partial_kernel(const De
         for (int i = threadIdx.x; i < DH + 2; i += kWarps * 32) out[i] = i == 0 ? -INFINITY : 0.f;
         return;
     }
-    const __nv_bfloat16* Kp = static_cast<const __nv_bfloat16*>(L.k) + b * L.sb + h * L.sh + sub * 8;
-    const __nv_bfloat16* Vp = static_cast<const __nv_bfloat16*>(L.v) + b * L.sb + h * L.sh + sub * 8;
+    const __nv_bfloat16* Kp = static_cast<const __nv_bfloat16*>(L.k) + b * L.sb + (h / p.kv_group) * L.sh + sub * 8;
+    const __nv_bfloat16* Vp = static_cast<const __nv_bfloat16*>(L.v) + b * L.sb + (h / p.kv_group) * L.sh + sub * 8;
 
     float q[8];
     {
@@ -336,6 +336,8 @@ extern "C" mka_status mka_decode_static(const mka_shape* s, const void* q, const
         p.n_chunks[l] = plan.n_chunks[l];
     }
     p.B = s->B; p.H = s->H; p.d = s->d;
+    if (s->kv_heads < 0 || (s->kv_heads > 0 && (s->H % s->kv_heads != 0))) return MKA_ERR_SHAPE;
+    p.kv_group = s->kv_heads > 0 ? s->H / s->kv_heads : 1;
     p.scale = s->scale > 0.f ? s->scale : 1.0f / sqrtf((float)s->d);
     p.chunk_rows = plan.chunk_rows;
     p.total_chunks = plan.total_chunks;

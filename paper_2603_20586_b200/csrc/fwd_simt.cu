@@ -59,8 +59,8 @@ __global__ void __launch_bounds__(kThreads) fwd_simt_kernel(const FwdParams p) {
         visible_range(lvl, t0 + p.q_offset, p.window, L.n, p.decode, lo_first, hi_first);
         visible_range(lvl, t_last + p.q_offset, p.window, L.n, p.decode, lo_last, hi_last);
         const long long lo = lo_first, hi = hi_last > hi_first ? hi_last : hi_first;
-        const T* Kp = static_cast<const T*>(L.k) + b * L.sb + h * L.sh;
-        const T* Vp = static_cast<const T*>(L.v) + b * L.sb + h * L.sh;
+        const T* Kp = static_cast<const T*>(L.k) + b * L.sb + (h / p.kv_group) * L.sh;
+        const T* Vp = static_cast<const T*>(L.v) + b * L.sb + (h / p.kv_group) * L.sh;
         float lam[kWarpRows];
         long long rlo[kWarpRows], rhi[kWarpRows];
 #pragma unroll

@@ -46,6 +46,7 @@ struct TcParams {
     const float* gate;
     long long n[3];
     int B, H, T;
+    int kv_group;            // query heads per KV head
     int window, q_offset;
     float scale_log2;
     unsigned int* status;
@@ -154,13 +155,13 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     mbar_expect_tx(&bar.k_full[s], C::kTileBytes);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes, &maps.k[l], pn * 64, kt * kTileN, h, b, &bar.k_full[s]);
+                        tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes, &maps.k[l], pn * 64, kt * kTileN, h / p.kv_group, b, &bar.k_full[s]);
                     ++issued_k;
                     if (!mbar_wait(&bar.v_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(&bar.v_full[s], C::kTileBytes);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes, &maps.v[l], pn * 64, kt * kTileN, h, b, &bar.v_full[s]);
+                        tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes, &maps.v[l], pn * 64, kt * kTileN, h / p.kv_group, b, &bar.v_full[s]);
                     ++issued_v;
                 }
             }
@@ -418,8 +419,8 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
         return cudaErrorNotSupported;
     for (int l = 0; l < 3; ++l) {
         if (fp.L[l].n == 0) { maps.k[l] = maps.q; maps.v[l] = maps.q; continue; }
-        if (!make_map(&maps.k[l], fp.L[l].k, DH, fp.L[l].n, fp.H, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb) ||
-            !make_map(&maps.v[l], fp.L[l].v, DH, fp.L[l].n, fp.H, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb))
+        if (!make_map(&maps.k[l], fp.L[l].k, DH, fp.L[l].n, fp.H / fp.kv_group, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb) ||
+            !make_map(&maps.v[l], fp.L[l].v, DH, fp.L[l].n, fp.H / fp.kv_group, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb))
             return cudaErrorNotSupported;
     }
     TcParams p;
@@ -427,7 +428,7 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
     p.LSE = fp.LSE;
     p.gate = fp.gate;
     for (int l = 0; l < 3; ++l) p.n[l] = fp.L[l].n;
-    p.B = fp.B; p.H = fp.H; p.T = fp.T;
+    p.B = fp.B; p.H = fp.H; p.T = fp.T; p.kv_group = fp.kv_group;
     p.window = fp.window; p.q_offset = fp.q_offset;
     p.scale_log2 = fp.scale * kLog2e;
     p.status = status_word;
@@ -449,7 +450,7 @@ bool fwd_tc_eligible(const FwdParams& p, int dtype) {
         if (L.n == 0) continue;
         if (L.n > 0x7fffffffLL) return false;
         if (L.sn % 8 || L.sn <= 0) return false;
-        if (p.H > 1 && (L.sh % 8 || L.sh <= 0)) return false;
+        if (p.H / (p.kv_group > 0 ? p.kv_group : 1) > 1 && (L.sh % 8 || L.sh <= 0)) return false;
         if (p.B > 1 && (L.sb % 8 || L.sb <= 0)) return false;
     }
     return tensor_map_encoder_available();

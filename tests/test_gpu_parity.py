@@ -5,6 +5,7 @@ import pytest
 import torch
 
 from gpu_helpers import check, err, np64, problem
+from mka_inputs import approx_normal
 
 pytestmark = pytest.mark.gpu
 
@@ -318,3 +319,42 @@ def test_workspace_too_small_is_rejected(mka):
     with pytest.raises(mka.MkaError) as e:
         mka.mka_decode(mka.make_shape(B, H, 1, d), q, [K, None, None], [K, None, None], gate, ws=ws)
     assert e.value.code == 4
+
+
+# ------------------------------------------------------------------ grouped-query heads (mka_shape.kv_heads)
+@pytest.mark.parametrize("d,flags", [(128, 0), (64, 0), (64, 1)])
+def test_fwd_and_decode_with_grouped_query_heads(mka, orc, d, flags):
+    """H query heads on H_kv KV heads: same result as the dense operator on the KV heads repeated per group."""
+    B, H, H_kv, T, W, N = 2, 6, 2, 300, 70, (300, 300, 96)
+    P = problem(41, B, H_kv, T, d, N, 64, torch.bfloat16)
+    Q = approx_normal(41, 50, 0, B * H * T * d, 1.0, "cpu", torch.bfloat16).view(B, H, T, d).cuda()
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    shape = mka.make_shape(B, H, T, d, 64, W, flags=flags, kv_heads=H_kv)
+    assert mka.mka_fwd_kernel_kind(shape, P["K"], P["V"]) == (0 if flags else 1)
+    O, LSE = mka.mka_fwd(shape, Q, P["K"], P["V"], gate)
+    G = H // H_kv
+    Kr = [np.repeat(np64(k), G, axis=1) for k in P["K"]]
+    Vr = [np.repeat(np64(v), G, axis=1) for v in P["V"]]
+    Or, Lr = orc.fwd(np64(Q), Kr, Vr, np64(gate), W)
+    check(O, Or, torch.bfloat16, "grouped-query fwd O")
+    assert np.abs(np64(LSE) - Lr).max() <= 2e-3
+    if not flags:
+        q1, g1 = Q[:, :, -1].contiguous(), gate[:, -1].contiguous()
+        Od, _ = mka.mka_decode(mka.make_shape(B, H, 1, d, 64, kv_heads=H_kv), q1, P["K"], P["V"], g1)
+        Odr, _ = orc.fwd(np64(q1)[:, :, None], Kr, Vr, np64(g1)[:, None], 1, decode=True)
+        check(Od.view(B, H, 1, d), Odr, torch.bfloat16, "grouped-query decode O")
+
+
+def test_grouped_query_heads_argument_checks(mka):
+    B, H, T, d = 1, 6, 128, 64
+    P = problem(42, B, 2, T, d, (128, 128, 64), 64, torch.bfloat16, with_dO=False)
+    Q = torch.zeros(B, H, T, d, dtype=torch.bfloat16, device="cuda")
+    gate = torch.full((B, T, 3), 1.0 / 3, device="cuda")
+    with pytest.raises(mka.MkaError) as e:                       # 6 heads do not split over 4 KV heads
+        mka.mka_fwd(mka.make_shape(B, H, T, d, 64, 32, kv_heads=4), Q, P["K"], P["V"], gate)
+    assert e.value.code == 2
+    O, LSE = mka.mka_fwd(mka.make_shape(B, H, T, d, 64, 32, kv_heads=2), Q, P["K"], P["V"], gate)
+    with pytest.raises(mka.MkaError) as e:                       # gradients of shared KV heads are not built
+        mka.mka_bwd(mka.make_shape(B, H, T, d, 64, 32, kv_heads=2), Q, P["K"], P["V"], gate, O, LSE, torch.zeros_like(Q),
+                    want_router_grad=False)
+    assert e.value.code == 5
