@@ -97,8 +97,9 @@ typedef struct mka_shape {
     uint32_t flags;  /* MKA_FLAG_* */
     int32_t kv_heads; /* grouped-query sharing (the paper evaluates on GQA models): 0 or H = one KV head per query
                          head; otherwise H % kv_heads == 0, the levels hold kv_heads heads ([B, kv_heads, n, d]) and
-                         query head h reads KV head h / (H / kv_heads).  Honoured by mka_fwd and mka_decode;
-                         mka_bwd returns MKA_ERR_UNSUPPORTED for kv_heads != H (the paged decode has its own H_kv) */
+                         query head h reads KV head h / (H / kv_heads).  Honoured by mka_fwd, mka_decode and
+                         the tensor-core path of mka_bwd (dK, dV then hold kv_heads heads, summed over each group;
+                         the CUDA-core backward returns MKA_ERR_UNSUPPORTED); the paged decode has its own H_kv */
 } mka_shape;
 
 /* Split table of the decode kernel: level l is cut into n_chunks[l] chunks of chunk_rows rows (the last

@@ -359,7 +359,6 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     mka_status st = check_shape(s, false);
     if (st != MKA_OK) return st;
     if (s->mode != MKA_MODE_FAST) return MKA_ERR_UNSUPPORTED;
-    if (kv_group_of(s) != 1) return MKA_ERR_UNSUPPORTED;      // gradients of shared KV heads: not built
     if ((st = check_levels(s, L)) != MKA_OK) return st;
     if (!dL) return MKA_ERR_ARG;
     for (int l = 0; l < 3; ++l) {
@@ -397,11 +396,13 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     w += round_up((size_t)kRouterBwdChunks * (s->D > 0 ? s->D : 0) * 3 * sizeof(float), 256);
     p.stats = reinterpret_cast<float*>(w);
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
-    p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s);
+    p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s); p.kv_group = kv_group_of(s);
+    const bool tc = !(s->flags & MKA_FLAG_FORCE_SIMT) && bwd_tc_eligible(p, s->dtype);
+    if (!tc && p.kv_group != 1) return MKA_ERR_UNSUPPORTED;   // shared KV heads: only the tensor-core kernels sum over a group
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
     cudaError_t e;
-    if (!(s->flags & MKA_FLAG_FORCE_SIMT) && bwd_tc_eligible(p, s->dtype))
+    if (tc)
         e = launch_bwd_tc(p, static_cast<unsigned int*>(ws), cs);
     else
         e = launch_bwd_simt(p, s->dtype, cs);
@@ -499,7 +500,7 @@ int32_t mka_bwd_kernel_kind(const mka_shape* s, const mka_level L[3], const mka_
         p.dL[l].sh = dL ? dL[l].stride_h : L[l].stride_h;
         p.dL[l].sb = dL ? dL[l].stride_b : L[l].stride_b;
     }
-    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.kv_group = kv_group_of(s);
     return (!(s->flags & MKA_FLAG_FORCE_SIMT) && bwd_tc_eligible(p, s->dtype)) ? 1 : 0;
 }
 

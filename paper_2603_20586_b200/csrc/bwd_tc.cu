@@ -51,6 +51,7 @@ struct BwdTcParams {
     LevelGradDev dL[3];
     long long n[3];
     int B, H, T, Tpad;
+    int kv_group;             // query heads per KV head: K, V, dK, dV hold H / kv_group heads
     int window, q_offset;
     float scale, scale_log2;
     int kv_tiles[3];          // 128-row key tiles per level
@@ -228,13 +229,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                     mbar_expect_tx(&bar.a_full[s], C::kTile);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sK + s * C::kTile + pn * kPanel, &maps.k[l], pn * 64, kt * kBlk, h, b, &bar.a_full[s]);
+                        tma_load_4d(sK + s * C::kTile + pn * kPanel, &maps.k[l], pn * 64, kt * kBlk, h / p.kv_group, b, &bar.a_full[s]);
                     ++issued_k;
                     if (!mbar_wait(&bar.b_empty[sv], phv ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(&bar.b_full[sv], C::kTile);
 #pragma unroll
                     for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sV + sv * C::kTile + pn * kPanel, &maps.v[l], pn * 64, kt * kBlk, h, b, &bar.b_full[sv]);
+                        tma_load_4d(sV + sv * C::kTile + pn * kPanel, &maps.v[l], pn * 64, kt * kBlk, h / p.kv_group, b, &bar.b_full[sv]);
                     ++issued_v;
                 }
             }
@@ -439,8 +440,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
-    const int b = blockIdx.z, h = blockIdx.y;
-    const long long bh = (long long)b * p.H + h;
+    const int b = blockIdx.z, h = blockIdx.y;               // h: KV head; its query heads are h * G .. h * G + G - 1
     // key tiles in decreasing order of work: L3 (seen by every query), L2 from the oldest key on, L1
     int lvl, kt;
     {
@@ -459,7 +459,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     if (t_lo < 0) t_lo = 0;
     if (t_hi > p.T) t_hi = p.T;
     const int first = t_hi > t_lo ? (int)(t_lo / kBlk) : 0;
-    const int E = t_hi > t_lo ? (int)((t_hi + kBlk - 1) / kBlk) - first : 0;
+    const int Eq = t_hi > t_lo ? (int)((t_hi + kBlk - 1) / kBlk) - first : 0;    // query tiles of ONE head that see this key tile
+    const int E = Eq * p.kv_group;                          // the stream: head by head, each head's tiles in order
 
     if (tid == 0) {
         abort_flag = 0;
@@ -489,22 +490,25 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                 tma_load_4d(sK + pn * kPanel, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
                 tma_load_4d(sV + pn * kPanel, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
             }
-            const float* statD = p.statD + bh * p.Tpad;
-            const float* statB = p.statB[lvl] + bh * p.Tpad;
+            int hq = h * p.kv_group, eq = 0;                // query head and tile-within-head of stage e
             for (int e = 0; e < E; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
                 if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) break;
-                const int tt = (first + e) * kBlk;
+                const long long bh = (long long)b * p.H + hq;
+                const float* statD = p.statD + bh * p.Tpad;
+                const float* statB = p.statB[lvl] + bh * p.Tpad;
+                const int tt = (first + eq) * kBlk;
                 mbar_expect_tx(&bar.a_full[s], 2 * C::kTile + C::kStatBytes);
 #pragma unroll
                 for (int pn = 0; pn < C::kPanels; ++pn) {
-                    tma_load_4d(sQ + s * C::kTile + pn * kPanel, &maps.q, pn * 64, tt, h, b, &bar.a_full[s]);
-                    tma_load_4d(sdO + s * C::kTile + pn * kPanel, &maps.dO, pn * 64, tt, h, b, &bar.a_full[s]);
+                    tma_load_4d(sQ + s * C::kTile + pn * kPanel, &maps.q, pn * 64, tt, hq, b, &bar.a_full[s]);
+                    tma_load_4d(sdO + s * C::kTile + pn * kPanel, &maps.dO, pn * 64, tt, hq, b, &bar.a_full[s]);
                 }
                 bulk_load(sStat + s * 2 * kBlk, statD + tt, kBlk * sizeof(float), &bar.a_full[s]);
                 bulk_load(sStat + s * 2 * kBlk + kBlk, statB + tt, kBlk * sizeof(float), &bar.a_full[s]);
                 ++issued;
+                if (++eq == Eq) { eq = 0; ++hq; }
             }
             mbar_wait(&bar.fixed_full, 0, abortp);
             for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
@@ -576,9 +580,11 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
         }
         const bool rows_full = j0 + kBlk - 1 < n;
         bool ok = true;
+        int eq = 0;                                                    // tile within the current query head
         for (int e = 0; e < E; ++e) {
             const int s = e % C::kStages;
-            const long long tt = (long long)(first + e) * kBlk;        // first query of the tile
+            const long long tt = (long long)(first + eq) * kBlk;       // first query of the tile
+            if (++eq == Eq) eq = 0;
             // The per-query statistics of the tile sit in this stage's shared memory; fetch this thread's 64 biases
             // before waiting for S so that the loads' latency (long while the tensor pipe saturates shared
             // memory) is off the path.  The stage's own barrier has long completed; waiting on it orders the reads.
@@ -703,7 +709,8 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
         p.n[l] = bp.L[l].n;
         p.kv_tiles[l] = (int)((bp.L[l].n + 127) / 128);
     }
-    p.B = bp.B; p.H = bp.H; p.T = bp.T; p.Tpad = Tpad;
+    p.B = bp.B; p.H = bp.H; p.T = bp.T; p.Tpad = Tpad; p.kv_group = bp.kv_group > 0 ? bp.kv_group : 1;
+    const int H_kv = bp.H / p.kv_group;
     p.window = bp.window; p.q_offset = bp.q_offset;
     p.scale = bp.scale; p.scale_log2 = bp.scale * kLog2e;
     p.status = status_word;
@@ -716,8 +723,8 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
             return cudaErrorNotSupported;
         for (int l = 0; l < 3; ++l) {
             if (bp.L[l].n == 0) { m.k[l] = m.q; m.v[l] = m.q; continue; }
-            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kBlk) ||
-                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kBlk))
+            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, H_kv, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kBlk) ||
+                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, H_kv, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, kBlk))
                 return cudaErrorNotSupported;
         }
         e = cudaFuncSetAttribute(bwd_dq_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemDq);
@@ -734,13 +741,13 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
             return cudaErrorNotSupported;
         for (int l = 0; l < 3; ++l) {
             if (bp.L[l].n == 0) { m.k[l] = m.q; m.v[l] = m.q; continue; }
-            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, 128) ||
-                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, bp.H, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, 128))
+            if (!make_bf16_map(&m.k[l], bp.L[l].k, DH, bp.L[l].n, H_kv, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, 128) ||
+                !make_bf16_map(&m.v[l], bp.L[l].v, DH, bp.L[l].n, H_kv, bp.B, bp.L[l].sn, bp.L[l].sh, bp.L[l].sb, 128))
                 return cudaErrorNotSupported;
         }
         e = cudaFuncSetAttribute(bwd_dkv_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemDkv);
         if (e != cudaSuccess) return e;
-        dim3 grid(tiles, bp.H, bp.B);
+        dim3 grid(tiles, H_kv, bp.B);
         bwd_dkv_tc_kernel<DH><<<grid, kThreads, C::kSmemDkv, st>>>(m, p);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -758,7 +765,7 @@ bool bwd_tc_eligible(const BwdParams& p, int dtype) {
         if (L.n == 0) continue;
         if (L.n > 0x7fffffffLL - 256) return false;
         if (L.sn % 8 || L.sn <= 0) return false;
-        if (p.H > 1 && (L.sh % 8 || L.sh <= 0)) return false;
+        if (p.H / (p.kv_group > 0 ? p.kv_group : 1) > 1 && (L.sh % 8 || L.sh <= 0)) return false;
         if (p.B > 1 && (L.sb % 8 || L.sb <= 0)) return false;
         if (p.dL[l].sn % 8 || p.dL[l].sh % 8 || p.dL[l].sb % 8) return false;
     }

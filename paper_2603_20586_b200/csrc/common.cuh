@@ -143,6 +143,7 @@ struct BwdParams {
     int B, H, T, d;
     int window, q_offset;
     float scale;
+    int kv_group;     // query heads per KV head (>= 1); > 1 only on the tensor-core path
 };
 cudaError_t launch_bwd_simt(const BwdParams& p, int dtype, cudaStream_t st);
 cudaError_t launch_router_bwd(const void* R, int r_dtype, const float* dG, long long rows, int D, float* dW_r,
