@@ -44,6 +44,9 @@ CASES = [
     PagedConfig("t_p1", 14, 2, 8, 2, 64, (33, 90, 17), 1, rows_frac=(1.0, 0.6)),         # one row per page
     PagedConfig("t_p256", 15, 2, 8, 4, 128, (300, 5000, 1000), 256, rows_frac=(0.9, 1.0)),
     PagedConfig("t_l2only", 16, 2, 6, 2, 128, (0, 1300, 0), 16),                         # absent levels
+    # many (sequence, KV head) groups make the split table pick chunks of more than 1024 rows; with one row per page a
+    # chunk then spans more table entries than the kernel keeps in shared memory (it looks them up in place)
+    PagedConfig("t_longchunk", 22, 8, 8, 8, 64, (0, 40000, 0), 1, rows_frac=(1.0, 0.93)),
 ]
 
 
