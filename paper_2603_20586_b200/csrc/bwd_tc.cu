@@ -90,43 +90,64 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
 __device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------ prep
-// One warp per padded row: D = dO . O and the three exponent biases.  Padding rows (t >= T) get a bias
-// of -inf so that a streamed sub-tile may run past the last query without a mask.
+// D = dO . O and the three exponent biases of every padded row.  DH / 8 lanes share a row (one 16-byte load of O and
+// one of dO each), a warp covers 2 or 4 rows per pass and a thread works on four passes at once, so eight loads are
+// in flight per thread.  Padding rows (t >= T) get a bias of -inf so that a streamed sub-tile may run past the last
+// query without a mask.
 template <int DH>
 __global__ void __launch_bounds__(256) bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
                                                        const float* __restrict__ LSE, const float* __restrict__ gate, int H,
                                                        int T, int Tpad, long long rows_pad, float* __restrict__ sD,
                                                        float* __restrict__ b0, float* __restrict__ b1, float* __restrict__ b2) {
-    const int lane = threadIdx.x & 31;
-    const long long r = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (r >= rows_pad) return;
-    const long long bh = r / Tpad;
-    const int t = (int)(r % Tpad);
-    float dsum = 0.f, o0 = -INFINITY, o1 = -INFINITY, o2 = -INFINITY;
-    if (t < T) {
-        const long long row = bh * T + t;
-        constexpr int PER = DH / 32;                   // 2 or 4 consecutive elements per lane
-        const __nv_bfloat16* po = O + row * DH + lane * PER;
-        const __nv_bfloat16* pg = dO + row * DH + lane * PER;
+    constexpr int LPR = DH / 8;                            // lanes per row: 16 or 8
+    constexpr int RPW = 32 / LPR;                          // rows per warp and pass
+    constexpr int kPasses = 4;
+    const int lane = threadIdx.x & 31, sub = lane % LPR, grp = lane / LPR;
+    const long long warp_row0 = ((long long)blockIdx.x * 8 + (threadIdx.x >> 5)) * (RPW * kPasses);
+    uint4 a[kPasses], g[kPasses];
+    long long rr[kPasses];
+    bool in[kPasses];
+#pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        rr[u] = warp_row0 + u * RPW + grp;
+        const long long bh = rr[u] / Tpad;
+        const int t = (int)(rr[u] % Tpad);
+        in[u] = rr[u] < rows_pad && t < T;
+        a[u] = g[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (in[u]) {
+            const long long off = (bh * T + t) * DH + sub * 8;
+            a[u] = __ldg(reinterpret_cast<const uint4*>(O + off));
+            g[u] = __ldg(reinterpret_cast<const uint4*>(dO + off));
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        const uint32_t aw[4] = {a[u].x, a[u].y, a[u].z, a[u].w}, gw[4] = {g[u].x, g[u].y, g[u].z, g[u].w};
         float s = 0.f;
 #pragma unroll
-        for (int i = 0; i < PER; i += 2) {
-            const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(po + i);
-            const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(pg + i);
-            s = fmaf(__bfloat162float(a.x), __bfloat162float(g.x), s);
-            s = fmaf(__bfloat162float(a.y), __bfloat162float(g.y), s);
+        for (int i = 0; i < 4; ++i) {
+            s = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(gw[i] << 16), s);
+            s = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(gw[i] & 0xffff0000u), s);
         }
-        s = warp_sum(s);
-        const float lse = LSE[row];
-        const float* g = gate + ((bh / H) * T + t) * 3;
-        const bool live = lse > -INFINITY;
-        const float l2 = lse * kLog2e;
-        dsum = s;
-        o0 = (live && g[0] > 0.f) ? log2f(g[0]) - l2 : -INFINITY;
-        o1 = (live && g[1] > 0.f) ? log2f(g[1]) - l2 : -INFINITY;
-        o2 = (live && g[2] > 0.f) ? log2f(g[2]) - l2 : -INFINITY;
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (sub == 0 && rr[u] < rows_pad) {
+            float o0 = -INFINITY, o1 = -INFINITY, o2 = -INFINITY;
+            if (in[u]) {
+                const long long bh = rr[u] / Tpad;
+                const int t = (int)(rr[u] % Tpad);
+                const float lse = LSE[bh * T + t];
+                const float* gt = gate + ((bh / H) * T + t) * 3;
+                const bool live = lse > -INFINITY;
+                const float l2 = lse * kLog2e;
+                o0 = (live && gt[0] > 0.f) ? log2f(gt[0]) - l2 : -INFINITY;
+                o1 = (live && gt[1] > 0.f) ? log2f(gt[1]) - l2 : -INFINITY;
+                o2 = (live && gt[2] > 0.f) ? log2f(gt[2]) - l2 : -INFINITY;
+            }
+            sD[rr[u]] = in[u] ? s : 0.f;
+            b0[rr[u]] = o0; b1[rr[u]] = o1; b2[rr[u]] = o2;
+        }
     }
-    if (lane == 0) { sD[r] = dsum; b0[r] = o0; b1[r] = o1; b2[r] = o2; }
 }
 
 // Key tile range [first, end) (128-row units) of query rows [r0, r1] on one level.
@@ -693,7 +714,8 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
     for (int l = 0; l < 3; ++l) statB[l] = bp.stats + (long long)(1 + l) * rows_pad;
     const long long sq_n = DH, sq_h = (long long)bp.T * DH, sq_b = (long long)bp.H * bp.T * DH;
 
-    bwd_prep_kernel<DH><<<(unsigned)((rows_pad + 7) / 8), 256, 0, st>>>(
+    constexpr int kPrepRowsPerBlock = 8 * (32 / (DH / 8)) * 4;          // 8 warps x rows per pass x passes
+    bwd_prep_kernel<DH><<<(unsigned)((rows_pad + kPrepRowsPerBlock - 1) / kPrepRowsPerBlock), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(bp.O), static_cast<const __nv_bfloat16*>(bp.dO), bp.LSE, bp.gate, bp.H, bp.T, Tpad,
         rows_pad, statD, statB[0], statB[1], statB[2]);
     cudaError_t e = cudaGetLastError();
