@@ -137,7 +137,7 @@ struct L3RetrieveParams {
     int B, H, H_kv, d, bits, R, page_rows, max_bank;
 };
 
-constexpr int kRetThreads = 256;
+constexpr int kRetThreads = 1024;
 constexpr int kMaxR = 64;
 constexpr unsigned short kTaken = 0xffffu;
 

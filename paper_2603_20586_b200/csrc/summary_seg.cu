@@ -352,7 +352,10 @@ cudaError_t launch_w(const void* X, SegParams p, cudaStream_t st) {
     CUtensorMap map;
     if (!make_strip_map(&map, X, sizeof(T) == 2, p.D, p.T, p.B, kNC, kSegBoxRows)) return cudaErrorNotSupported;
     const size_t smem = (size_t)kSegTileBytes + 128;
-    cudaError_t e = cudaFuncSetAttribute(l2_summary_seg_kernel<T, kEma, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // the ticket counter and the records this launch will use start at zero
+    cudaError_t e = cudaMemsetAsync(p.ticket, 0, 256 + (size_t)p.B * p.S * p.D * sizeof(unsigned long long), st);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(l2_summary_seg_kernel<T, kEma, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const long long resident = (long long)kSegCtasPerSm * 148;
     l2_summary_seg_kernel<T, kEma, WB><<<(unsigned)(tiles < resident ? tiles : resident), kSegThreads, smem, st>>>(map, p);
@@ -386,8 +389,6 @@ cudaError_t launch_l2_summary_seg(const void* X, void* M2, float* state, int use
     p.rec = reinterpret_cast<unsigned long long*>(static_cast<char*>(scratch) + 256);
     p.M2 = M2; p.state = state; p.T = T; p.n_prev = n_prev; p.B = B; p.D = D; p.kind = kind; p.beta = beta;
     p.use_state = use_state; p.status = status;
-    cudaError_t e = cudaMemsetAsync(scratch, 0, l2_summary_seg_workspace(B, T, D, dtype), st);
-    if (e != cudaSuccess) return e;
     if (dtype == MKA_F32) return kind == MKA_SUMMARY_EMA ? launch_k<float, true>(X, p, st) : launch_k<float, false>(X, p, st);
     return kind == MKA_SUMMARY_EMA ? launch_k<__nv_bfloat16, true>(X, p, st) : launch_k<__nv_bfloat16, false>(X, p, st);
 }
