@@ -175,6 +175,7 @@ typedef struct mka_paged_level {
                                    b*table_stride + h*table_head_stride (per-head recall lists of mka_l3_retrieve) */
     int32_t page_rows;          /* rows per page: a power of two */
     int64_t stride_page, stride_h, stride_n;
+    int64_t pool_pages;         /* pages in the pool; read by mka_fwd_paged only (mka_decode_paged ignores it) */
 } mka_paged_level;
 
 /*
@@ -188,6 +189,16 @@ typedef struct mka_paged_level {
  *       chunks of a multiple of 128 rows (at most 8192), chosen so that the grid makes few rounds of the resident CTAs
  * d must be 64 or 128; pools 16-byte aligned with strides that are multiples of 8 elements.
  */
+/*
+ * Fused forward of mka_fwd over paged levels (prefill, or a chunk of it, against a paged KV cache) with grouped-query
+ * sharing: same result as mka_fwd on the gathered levels with shape->kv_heads = H_kv.  Every sequence has L[l].n
+ * rows on level l (rows must be NULL); page_rows must be a power of two >= 8; pool_pages must be set; rows of a
+ * sequence's last page past n must hold finite values (they are loaded and masked, not skipped).
+ * bf16, MKA_MODE_FAST, d in {64, 128} only (the TMA + tcgen05 kernel; a 128-row key tile is assembled from one box
+ * per page); anything else returns MKA_ERR_UNSUPPORTED.  ws: at least 256 bytes (status word).
+ */
+mka_status mka_fwd_paged(const mka_shape* shape, int32_t H_kv, const void* Q, const mka_paged_level L[3],
+                         const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
 size_t mka_decode_paged_workspace_bytes(const mka_shape* shape, int32_t H_kv, const int64_t n_level[3]);
 mka_status mka_decode_paged(const mka_shape* shape, int32_t H_kv, const void* q, const mka_paged_level L[3],
                             const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);

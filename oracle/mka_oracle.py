@@ -418,3 +418,37 @@ def l3_retrieve(q, proj, codes, bank, bank_len, R: int, H_kv: int):
             table[b, h, :len(pos)] = pages[pos]
             n_sel[b] = len(pos)
     return table, n_sel
+
+
+def fwd_paged(Q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, n: Sequence[int], page_rows: int, gate,
+              window: int, q_offset: int = 0, scale: Optional[float] = None):
+    """Forward of the operator over paged levels with grouped-query sharing: every sequence's levels (n[l] rows each)
+    are gathered through the page tables, the KV heads repeated over their groups, and the dense forward does the rest.
+    Q [B, H, T, d]; pools [P_l, H_kv, page_rows, d] or None; tables[l] [B, pages] or [B, H_kv, pages]; gate [B, T, 3]."""
+    Q = _f64(Q)
+    gate = _f64(gate)
+    B, H, T, d = Q.shape
+    O = np.empty((B, H, T, d))
+    LSE = np.empty((B, H, T))
+    for b in range(B):
+        Ks, Vs = [], []
+        for l in range(3):
+            if pools_k[l] is None or int(n[l]) == 0:
+                Ks.append(np.zeros((1, H, 0, d)))
+                Vs.append(np.zeros((1, H, 0, d)))
+                continue
+            pk, pv = _f64(pools_k[l]), _f64(pools_v[l])
+            H_kv = pk.shape[1]
+            tab = np.asarray(tables[l][b])
+            if tab.ndim == 2:
+                kd = np.concatenate([gather_pages(pk[:, h:h + 1], tab[h], int(n[l]), page_rows) for h in range(H_kv)], axis=0)
+                vd = np.concatenate([gather_pages(pv[:, h:h + 1], tab[h], int(n[l]), page_rows) for h in range(H_kv)], axis=0)
+            else:
+                kd = gather_pages(pk, tab, int(n[l]), page_rows)
+                vd = gather_pages(pv, tab, int(n[l]), page_rows)
+            share = np.arange(H) // (H // H_kv)
+            Ks.append(kd[share][None])
+            Vs.append(vd[share][None])
+        o, ls = fwd(Q[b:b + 1], Ks, Vs, gate[b:b + 1], window, q_offset=q_offset, scale=scale)
+        O[b], LSE[b] = o[0], ls[0]
+    return O, LSE

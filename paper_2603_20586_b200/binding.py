@@ -26,7 +26,7 @@ TILE = 128
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
            "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_l2_summary_workspace_bytes", "mka_l2_summary_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes",
-           "mka_decode_paged", "mka_decode_paged_workspace_bytes", "mka_l3_index", "mka_l3_retrieve"]
+           "mka_decode_paged", "mka_decode_paged_workspace_bytes", "mka_l3_index", "mka_l3_retrieve", "mka_fwd_paged"]
 
 
 class MkaError(RuntimeError):
@@ -49,7 +49,7 @@ class mka_paged_level(ctypes.Structure):
     _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("page_table", ctypes.c_void_p),
                 ("rows", ctypes.c_void_p), ("n", ctypes.c_int64), ("table_stride", ctypes.c_int64),
                 ("table_head_stride", ctypes.c_int64), ("page_rows", ctypes.c_int32), ("stride_page", ctypes.c_int64), ("stride_h", ctypes.c_int64),
-                ("stride_n", ctypes.c_int64)]
+                ("stride_n", ctypes.c_int64), ("pool_pages", ctypes.c_int64)]
 
 
 class mka_shape(ctypes.Structure):
@@ -98,6 +98,7 @@ def _load() -> ctypes.CDLL:
     lib.mka_decode_paged_workspace_bytes.argtypes = [ctypes.POINTER(mka_shape), i32, ctypes.POINTER(ctypes.c_int64)]
     lib.mka_decode_paged.argtypes = [ctypes.POINTER(mka_shape), i32, vp, ctypes.POINTER(mka_paged_level), vp, vp, vp, vp,
                                      ctypes.c_size_t, vp]
+    lib.mka_fwd_paged.argtypes = lib.mka_decode_paged.argtypes
     lib.mka_l3_index.argtypes = [vp, i64, i32, i32, i32, i64, i64, i64, vp, i32, vp, vp]
     lib.mka_l3_retrieve.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.mka_l2_summary_kernel_kind.argtypes = [i32, i64, i32, i32, ctypes.c_size_t]
@@ -230,7 +231,7 @@ def _paged_levels(pools_k, pools_v, tables, rows, n):
     for l in range(3):
         k, v = pools_k[l], pools_v[l]
         if k is None or n[l] == 0:
-            arr[l] = mka_paged_level(None, None, None, None, 0, 0, 0, 1, 0, 0, 0)
+            arr[l] = mka_paged_level(None, None, None, None, 0, 0, 0, 1, 0, 0, 0, 0)
             continue
         # pools [pages, H_kv, page_rows, d]; any strides with d contiguous
         assert k.dim() == 4 and k.stride(3) == 1 and v.stride() == k.stride() and v.shape == k.shape
@@ -240,8 +241,24 @@ def _paged_levels(pools_k, pools_v, tables, rows, n):
         r = None if rows is None else rows[l]
         assert r is None or (r.dtype == torch.int32 and r.is_contiguous())
         arr[l] = mka_paged_level(k.data_ptr(), v.data_ptr(), tab.data_ptr(), _ptr(r), int(n[l]), tab.stride(0),
-                                 tab.stride(1) if tab.dim() == 3 else 0, k.shape[2], k.stride(0), k.stride(1), k.stride(2))
+                                 tab.stride(1) if tab.dim() == 3 else 0, k.shape[2], k.stride(0), k.stride(1), k.stride(2),
+                                 k.shape[0])
     return arr
+
+
+def mka_fwd_paged(shape: mka_shape, H_kv: int, Q, pools_k, pools_v, tables, n, gate, O=None, LSE=None, ws=None, stream=None):
+    """mka_fwd over paged levels with grouped-query head sharing (every sequence has n[l] rows on level l)."""
+    assert Q.is_contiguous() and gate.is_contiguous() and gate.dtype == torch.float32
+    B, H, T, d = Q.shape
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None:
+        LSE = torch.empty(B, H, T, dtype=torch.float32, device=Q.device)
+    if ws is None:
+        ws = torch.zeros(256, dtype=torch.uint8, device=Q.device)
+    _check(lib.mka_fwd_paged(ctypes.byref(shape), H_kv, _ptr(Q), _paged_levels(pools_k, pools_v, tables, None, n), _ptr(gate),
+                             _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream)), "mka_fwd_paged")
+    return O, LSE
 
 
 def mka_decode_paged_workspace_bytes(shape: mka_shape, H_kv: int, n) -> int:

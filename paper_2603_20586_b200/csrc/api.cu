@@ -255,6 +255,56 @@ static mka_status paged_plan(const int64_t n_level[3], int32_t B, int32_t H_kv, 
     return MKA_OK;
 }
 
+mka_status mka_fwd_paged(const mka_shape* s, int32_t H_kv, const void* Q, const mka_paged_level L[3], const float* gate,
+                         void* O, float* LSE, void* ws, size_t ws_bytes, void* stream) {
+    mka_status st = check_shape(s, false);
+    if (st != MKA_OK) return st;
+    if (s->dtype != MKA_BF16 || s->mode != MKA_MODE_FAST || (s->flags & MKA_FLAG_FORCE_SIMT)) return MKA_ERR_UNSUPPORTED;
+    if (s->d != 64 && s->d != 128) return MKA_ERR_UNSUPPORTED;
+    if (!L) return MKA_ERR_ARG;
+    if (H_kv <= 0 || (s->H > 0 && s->H % H_kv != 0)) return MKA_ERR_SHAPE;
+    if (s->H > 65535 || s->B > 65535) return MKA_ERR_SHAPE;
+    FwdParams p;
+    memset(&p, 0, sizeof(p));
+    PagedLevelDev P[3];
+    memset(P, 0, sizeof(P));
+    for (int l = 0; l < 3; ++l) {
+        if (L[l].n < 0 || L[l].n > 0x7fffffffLL) return MKA_ERR_SHAPE;
+        p.L[l].n = L[l].n;
+        if (L[l].n == 0) continue;
+        if (!L[l].k || !L[l].v || !L[l].page_table) return MKA_ERR_ARG;
+        if (L[l].rows) return MKA_ERR_UNSUPPORTED;                 // one length for all sequences
+        const int pr = L[l].page_rows;
+        if (pr < 8 || (pr & (pr - 1)) != 0) return MKA_ERR_SHAPE;
+        if (L[l].pool_pages <= 0 || L[l].pool_pages > 0x7fffffffLL || L[l].table_head_stride < 0) return MKA_ERR_SHAPE;
+        const int64_t width = L[l].table_head_stride > 0 ? L[l].table_head_stride : L[l].table_stride;
+        if (width * pr < L[l].n) return MKA_ERR_SHAPE;
+        if (L[l].stride_n < s->d || L[l].stride_page <= 0 || L[l].stride_h < 0) return MKA_ERR_SHAPE;
+        if (!aligned16(L[l].k) || !aligned16(L[l].v)) return MKA_ERR_ALIGN;
+        if (L[l].stride_n % 8 || L[l].stride_page % 8 || L[l].stride_h % 8) return MKA_ERR_ALIGN;
+        if (H_kv > 1 && L[l].stride_h <= 0) return MKA_ERR_SHAPE;
+        int shift = 0;
+        while ((1 << shift) < pr) ++shift;
+        P[l].k = L[l].k; P[l].v = L[l].v; P[l].table = L[l].page_table; P[l].n = L[l].n;
+        P[l].table_stride = L[l].table_stride; P[l].table_head_stride = L[l].table_head_stride;
+        P[l].sp = L[l].stride_page; P[l].sh = L[l].stride_h; P[l].sn = L[l].stride_n;
+        P[l].pool_pages = L[l].pool_pages; P[l].page_shift = shift;
+    }
+    if (s->B == 0 || s->H == 0 || s->T == 0) return MKA_OK;
+    if (!Q || !gate || !O) return MKA_ERR_ARG;
+    if (!aligned16(Q) || !aligned16(O)) return MKA_ERR_ALIGN;
+    if (!ws || ws_bytes < kWsHeader) return MKA_ERR_WORKSPACE;
+    p.Q = Q; p.O = O; p.LSE = LSE; p.gate = gate;
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
+    p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s);
+    p.mode = s->mode; p.decode = 0; p.kv_group = s->H / H_kv; p.paged = P;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
+    cudaError_t e = launch_fwd_tc(p, static_cast<unsigned int*>(ws), cs);
+    if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
 size_t mka_decode_paged_workspace_bytes(const mka_shape* s, int32_t H_kv, const int64_t n_level[3]) {
     if (!s || !n_level || H_kv <= 0 || s->B < 0 || s->H < 0 || s->d <= 0) return 0;
     mka_decode_plan_t plan;

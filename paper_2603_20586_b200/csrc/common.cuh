@@ -31,6 +31,7 @@ struct LevelGradDev {
     long long n, sb, sh, sn;
 };
 
+struct PagedLevelDev;
 struct FwdParams {
     const void* Q;
     void* O;
@@ -43,6 +44,7 @@ struct FwdParams {
     int mode;
     int decode;         // every row visible
     int kv_group;       // query heads per KV head (>= 1): head h reads KV head h / kv_group
+    const PagedLevelDev* paged;   // host array of 3, or null: the levels are page pools (tensor-core forward only; L[l].n still holds the rows)
 };
 
 template <typename T> struct Elem;
@@ -109,6 +111,7 @@ struct PagedLevelDev {
     const int* table;    // [B, table_stride]
     const int* rows;     // [B] or null
     long long n, table_stride, table_head_stride, sp, sh, sn;
+    long long pool_pages; // pages in the pool (needed by the paged forward only)
     int page_shift;      // log2(page_rows)
 };
 struct DecodePagedParams {

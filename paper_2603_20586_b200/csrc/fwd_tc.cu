@@ -50,6 +50,11 @@ struct TcParams {
     int window, q_offset;
     float scale_log2;
     unsigned int* status;
+    // paged levels: a 128-row key tile is assembled from boxes of box_rows rows, one page-table look-up per box
+    int paged;
+    const int* table[3];
+    long long table_stride[3], table_head_stride[3];
+    int page_shift[3], box_rows[3], pool_pages[3];
 };
 
 template <int DH>
@@ -85,7 +90,7 @@ __device__ __forceinline__ void tile_range(int level, long long r0, long long r1
     end = (int)((hi + kTileN - 1) / kTileN);
 }
 
-template <int DH>
+template <int DH, bool kPaged>
 __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     using C = Cfg<DH>;
     extern __shared__ uint8_t smem_raw[];
@@ -146,22 +151,53 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     tma_load_4d(sQ + q * C::kTileBytes + pn * kPanelBytes, &maps.q, pn * 64, (int)(m0 + q * kTileM), h, b, &bar.q_full);
             int issued_k = 0, issued_v = 0;
             bool ok = true;
+            const int kvh = h / p.kv_group;
             for (int l = 0; l < 3 && ok; ++l) {
+                const int* tab = kPaged ? p.table[l] + (long long)b * p.table_stride[l] + (long long)kvh * p.table_head_stride[l] : nullptr;
                 for (int kt = first[l]; kt < end[l]; ++kt) {
                     const int e = issued_k;
                     const int s = e % C::kStages;
                     const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                    // paged: the pool page of every box of this tile (K and V share them); a box past the level's last
+                    // row is aimed past the pool, where the copy engine fills zeros as it does past a dense level's end
+                    int page[16];
+                    int n_box = 0, rpb = kTileN, in_mask = 0;
+                    if (kPaged) {
+                        rpb = p.box_rows[l];
+                        n_box = kTileN / rpb;
+                        in_mask = (1 << p.page_shift[l]) - 1;
+                        for (int bx = 0; bx < n_box; ++bx) {
+                            const long long row = (long long)kt * kTileN + bx * rpb;
+                            page[bx] = row < p.n[l] ? tab[row >> p.page_shift[l]] : p.pool_pages[l];
+                        }
+                    }
                     if (!mbar_wait(&bar.k_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(&bar.k_full[s], C::kTileBytes);
+                    if (!kPaged) {
 #pragma unroll
-                    for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes, &maps.k[l], pn * 64, kt * kTileN, h / p.kv_group, b, &bar.k_full[s]);
+                        for (int pn = 0; pn < C::kPanels; ++pn)
+                            tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes, &maps.k[l], pn * 64, kt * kTileN, kvh, b, &bar.k_full[s]);
+                    } else {
+                        for (int bx = 0; bx < n_box; ++bx)
+#pragma unroll
+                            for (int pn = 0; pn < C::kPanels; ++pn)
+                                tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes + bx * rpb * 128, &maps.k[l], pn * 64,
+                                            (kt * kTileN + bx * rpb) & in_mask, kvh, page[bx], &bar.k_full[s]);
+                    }
                     ++issued_k;
                     if (!mbar_wait(&bar.v_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(&bar.v_full[s], C::kTileBytes);
+                    if (!kPaged) {
 #pragma unroll
-                    for (int pn = 0; pn < C::kPanels; ++pn)
-                        tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes, &maps.v[l], pn * 64, kt * kTileN, h / p.kv_group, b, &bar.v_full[s]);
+                        for (int pn = 0; pn < C::kPanels; ++pn)
+                            tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes, &maps.v[l], pn * 64, kt * kTileN, kvh, b, &bar.v_full[s]);
+                    } else {
+                        for (int bx = 0; bx < n_box; ++bx)
+#pragma unroll
+                            for (int pn = 0; pn < C::kPanels; ++pn)
+                                tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes + bx * rpb * 128, &maps.v[l], pn * 64,
+                                            (kt * kTileN + bx * rpb) & in_mask, kvh, page[bx], &bar.v_full[s]);
+                    }
                     ++issued_v;
                 }
             }
@@ -417,13 +453,27 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
     TcMaps maps;
     if (!make_map(&maps.q, fp.Q, DH, fp.T, fp.H, fp.B, DH, (long long)fp.T * DH, (long long)fp.H * fp.T * DH))
         return cudaErrorNotSupported;
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.paged = fp.paged ? 1 : 0;
     for (int l = 0; l < 3; ++l) {
         if (fp.L[l].n == 0) { maps.k[l] = maps.q; maps.v[l] = maps.q; continue; }
+        if (fp.paged) {
+            // the pool as a [pages, KV heads, rows of a page, d] tensor; a box = (up to 128) rows of one page
+            const PagedLevelDev& P = fp.paged[l];
+            const int page_rows = 1 << P.page_shift;
+            const int rpb = page_rows < kTileN ? page_rows : kTileN;
+            if (!make_bf16_map(&maps.k[l], P.k, DH, page_rows, fp.H / fp.kv_group, (int)P.pool_pages, P.sn, P.sh, P.sp, rpb) ||
+                !make_bf16_map(&maps.v[l], P.v, DH, page_rows, fp.H / fp.kv_group, (int)P.pool_pages, P.sn, P.sh, P.sp, rpb))
+                return cudaErrorNotSupported;
+            p.table[l] = P.table; p.table_stride[l] = P.table_stride; p.table_head_stride[l] = P.table_head_stride;
+            p.page_shift[l] = P.page_shift; p.box_rows[l] = rpb; p.pool_pages[l] = (int)P.pool_pages;
+            continue;
+        }
         if (!make_map(&maps.k[l], fp.L[l].k, DH, fp.L[l].n, fp.H / fp.kv_group, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb) ||
             !make_map(&maps.v[l], fp.L[l].v, DH, fp.L[l].n, fp.H / fp.kv_group, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb))
             return cudaErrorNotSupported;
     }
-    TcParams p;
     p.O = static_cast<__nv_bfloat16*>(fp.O);
     p.LSE = fp.LSE;
     p.gate = fp.gate;
@@ -432,10 +482,11 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
     p.window = fp.window; p.q_offset = fp.q_offset;
     p.scale_log2 = fp.scale * kLog2e;
     p.status = status_word;
-    cudaError_t e = cudaFuncSetAttribute(fwd_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<DH>::kSmemBytes);
+    auto kern = fp.paged ? fwd_tc_kernel<DH, true> : fwd_tc_kernel<DH, false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<DH>::kSmemBytes);
     if (e != cudaSuccess) return e;
     dim3 grid((fp.T + kNumQ * kTileM - 1) / (kNumQ * kTileM), fp.H, fp.B);
-    fwd_tc_kernel<DH><<<grid, kThreads, Cfg<DH>::kSmemBytes, st>>>(maps, p);
+    kern<<<grid, kThreads, Cfg<DH>::kSmemBytes, st>>>(maps, p);
     return cudaGetLastError();
 }
 

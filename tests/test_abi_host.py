@@ -34,7 +34,7 @@ def test_struct_sizes_match_header_layout(mka):
     b = mka.binding
     assert ctypes.sizeof(b.mka_level) == 48 and ctypes.sizeof(b.mka_level_grad) == 48
     assert ctypes.sizeof(b.mka_shape) == 48                       # twelve 4-byte fields, kv_heads last
-    assert ctypes.sizeof(b.mka_paged_level) == 88                 # 4 pointers, 3 int64, int32 + padding, 3 int64
+    assert ctypes.sizeof(b.mka_paged_level) == 96                 # 4 pointers, 3 int64, int32 + padding, 4 int64
     assert ctypes.sizeof(b.mka_decode_plan_t) == 40 and ctypes.sizeof(b.mka_tile_range) == 32
 
 

@@ -105,3 +105,19 @@ def test_per_head_tables_that_agree_equal_the_shared_table(orc):
     O3, _ = orc.decode_paged(q, pk, pv, per_head, rows, pr, g)
     assert np.array_equal(O3[0, :2], O1[0, :2]) and not np.array_equal(O3[0, 2:], O1[0, 2:])
     assert np.array_equal(O3[1], O1[1])
+
+
+def test_paged_forward_with_identity_tables_is_the_dense_forward(orc):
+    rng = np.random.default_rng(9)
+    B, H, T, d, pr, n, W = 2, 2, 10, 8, 4, 12, 5
+    K = [rng.normal(size=(B, H, n, d)) for _ in range(3)]
+    V = [rng.normal(size=(B, H, n, d)) for _ in range(3)]
+    Q = rng.normal(size=(B, H, T, d))
+    g = rng.random((B, T, 3)) + 0.1
+    g /= g.sum(-1, keepdims=True)
+    pk = [k.reshape(B, H, n // pr, pr, d).transpose(0, 2, 1, 3, 4).reshape(B * n // pr, H, pr, d) for k in K]
+    pv = [v.reshape(B, H, n // pr, pr, d).transpose(0, 2, 1, 3, 4).reshape(B * n // pr, H, pr, d) for v in V]
+    tab = [np.arange(B * n // pr, dtype=np.int32).reshape(B, n // pr)] * 3
+    O, L = orc.fwd_paged(Q, pk, pv, tab, [n, n, n], pr, g, W, q_offset=2)
+    Od, Ld = orc.fwd(Q, K, V, g, W, q_offset=2)
+    assert np.array_equal(O, Od) and np.array_equal(L, Ld)
