@@ -191,9 +191,10 @@ typedef struct mka_paged_level {
  */
 /*
  * Fused forward of mka_fwd over paged levels (prefill, or a chunk of it, against a paged KV cache) with grouped-query
- * sharing: same result as mka_fwd on the gathered levels with shape->kv_heads = H_kv.  Every sequence has L[l].n
- * rows on level l (rows must be NULL); page_rows must be a power of two >= 8; pool_pages must be set; rows of a
- * sequence's last page past n must hold finite values (they are loaded and masked, not skipped).
+ * sharing: same result as mka_fwd on the gathered levels with shape->kv_heads = H_kv.  Sequence b has rows[b] rows on
+ * level l (L[l].n for all when rows is NULL); all sequences share T and q_offset.  page_rows must be a power of two
+ * >= 8; pool_pages must be set; rows of a sequence's last page past its length must hold finite values (they are
+ * loaded and masked, not skipped).
  * bf16, MKA_MODE_FAST, d in {64, 128} only (the TMA + tcgen05 kernel; a 128-row key tile is assembled from one box
  * per page); anything else returns MKA_ERR_UNSUPPORTED.  ws: at least 256 bytes (status word).
  */

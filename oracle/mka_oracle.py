@@ -424,7 +424,8 @@ def fwd_paged(Q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, n: Sequ
               window: int, q_offset: int = 0, scale: Optional[float] = None):
     """Forward of the operator over paged levels with grouped-query sharing: every sequence's levels (n[l] rows each)
     are gathered through the page tables, the KV heads repeated over their groups, and the dense forward does the rest.
-    Q [B, H, T, d]; pools [P_l, H_kv, page_rows, d] or None; tables[l] [B, pages] or [B, H_kv, pages]; gate [B, T, 3]."""
+    Q [B, H, T, d]; pools [P_l, H_kv, page_rows, d] or None; tables[l] [B, pages] or [B, H_kv, pages]; gate [B, T, 3];
+    n[l]: rows of level l, one number for all sequences or an array [B]."""
     Q = _f64(Q)
     gate = _f64(gate)
     B, H, T, d = Q.shape
@@ -433,7 +434,8 @@ def fwd_paged(Q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, n: Sequ
     for b in range(B):
         Ks, Vs = [], []
         for l in range(3):
-            if pools_k[l] is None or int(n[l]) == 0:
+            n_b = int(np.asarray(n[l]).reshape(-1)[b if np.ndim(n[l]) else 0])
+            if pools_k[l] is None or n_b == 0:
                 Ks.append(np.zeros((1, H, 0, d)))
                 Vs.append(np.zeros((1, H, 0, d)))
                 continue
@@ -441,11 +443,11 @@ def fwd_paged(Q, pools_k: Sequence, pools_v: Sequence, tables: Sequence, n: Sequ
             H_kv = pk.shape[1]
             tab = np.asarray(tables[l][b])
             if tab.ndim == 2:
-                kd = np.concatenate([gather_pages(pk[:, h:h + 1], tab[h], int(n[l]), page_rows) for h in range(H_kv)], axis=0)
-                vd = np.concatenate([gather_pages(pv[:, h:h + 1], tab[h], int(n[l]), page_rows) for h in range(H_kv)], axis=0)
+                kd = np.concatenate([gather_pages(pk[:, h:h + 1], tab[h], n_b, page_rows) for h in range(H_kv)], axis=0)
+                vd = np.concatenate([gather_pages(pv[:, h:h + 1], tab[h], n_b, page_rows) for h in range(H_kv)], axis=0)
             else:
-                kd = gather_pages(pk, tab, int(n[l]), page_rows)
-                vd = gather_pages(pv, tab, int(n[l]), page_rows)
+                kd = gather_pages(pk, tab, n_b, page_rows)
+                vd = gather_pages(pv, tab, n_b, page_rows)
             share = np.arange(H) // (H // H_kv)
             Ks.append(kd[share][None])
             Vs.append(vd[share][None])

@@ -246,8 +246,10 @@ def _paged_levels(pools_k, pools_v, tables, rows, n):
     return arr
 
 
-def mka_fwd_paged(shape: mka_shape, H_kv: int, Q, pools_k, pools_v, tables, n, gate, O=None, LSE=None, ws=None, stream=None):
-    """mka_fwd over paged levels with grouped-query head sharing (every sequence has n[l] rows on level l)."""
+def mka_fwd_paged(shape: mka_shape, H_kv: int, Q, pools_k, pools_v, tables, n, gate, rows=None, O=None, LSE=None, ws=None,
+                  stream=None):
+    """mka_fwd over paged levels with grouped-query head sharing (n[l]: upper bound of the rows on level l; rows[l]:
+    int32 [B] rows of every sequence, or None)."""
     assert Q.is_contiguous() and gate.is_contiguous() and gate.dtype == torch.float32
     B, H, T, d = Q.shape
     if O is None:
@@ -256,7 +258,7 @@ def mka_fwd_paged(shape: mka_shape, H_kv: int, Q, pools_k, pools_v, tables, n, g
         LSE = torch.empty(B, H, T, dtype=torch.float32, device=Q.device)
     if ws is None:
         ws = torch.zeros(256, dtype=torch.uint8, device=Q.device)
-    _check(lib.mka_fwd_paged(ctypes.byref(shape), H_kv, _ptr(Q), _paged_levels(pools_k, pools_v, tables, None, n), _ptr(gate),
+    _check(lib.mka_fwd_paged(ctypes.byref(shape), H_kv, _ptr(Q), _paged_levels(pools_k, pools_v, tables, rows, n), _ptr(gate),
                              _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream)), "mka_fwd_paged")
     return O, LSE
 

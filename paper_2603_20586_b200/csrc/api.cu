@@ -273,7 +273,6 @@ mka_status mka_fwd_paged(const mka_shape* s, int32_t H_kv, const void* Q, const 
         p.L[l].n = L[l].n;
         if (L[l].n == 0) continue;
         if (!L[l].k || !L[l].v || !L[l].page_table) return MKA_ERR_ARG;
-        if (L[l].rows) return MKA_ERR_UNSUPPORTED;                 // one length for all sequences
         const int pr = L[l].page_rows;
         if (pr < 8 || (pr & (pr - 1)) != 0) return MKA_ERR_SHAPE;
         if (L[l].pool_pages <= 0 || L[l].pool_pages > 0x7fffffffLL || L[l].table_head_stride < 0) return MKA_ERR_SHAPE;
@@ -285,7 +284,7 @@ mka_status mka_fwd_paged(const mka_shape* s, int32_t H_kv, const void* Q, const 
         if (H_kv > 1 && L[l].stride_h <= 0) return MKA_ERR_SHAPE;
         int shift = 0;
         while ((1 << shift) < pr) ++shift;
-        P[l].k = L[l].k; P[l].v = L[l].v; P[l].table = L[l].page_table; P[l].n = L[l].n;
+        P[l].k = L[l].k; P[l].v = L[l].v; P[l].table = L[l].page_table; P[l].n = L[l].n; P[l].rows = L[l].rows;
         P[l].table_stride = L[l].table_stride; P[l].table_head_stride = L[l].table_head_stride;
         P[l].sp = L[l].stride_page; P[l].sh = L[l].stride_h; P[l].sn = L[l].stride_n;
         P[l].pool_pages = L[l].pool_pages; P[l].page_shift = shift;

@@ -55,6 +55,7 @@ struct TcParams {
     const int* table[3];
     long long table_stride[3], table_head_stride[3];
     int page_shift[3], box_rows[3], pool_pages[3];
+    const int* rows[3];      // per-sequence rows of a level (clamped to [0, n]), or null
 };
 
 template <int DH>
@@ -132,11 +133,21 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     const uint32_t tmem = tmem_base_slot;
     volatile int* abortp = &abort_flag;
 
+    // rows of the three levels for this sequence
+    long long nl[3];
+#pragma unroll
+    for (int l = 0; l < 3; ++l) {
+        nl[l] = p.n[l];
+        if (kPaged && p.rows[l]) {
+            const long long r = p.rows[l][b];
+            nl[l] = r < 0 ? 0 : (r < p.n[l] ? r : p.n[l]);
+        }
+    }
     // the CTA's level-ordered key-tile list (same closed form in every role)
     int first[3], end[3];
 #pragma unroll
     for (int l = 0; l < 3; ++l) {
-        if (p.n[l] > 0) tile_range(l, m0, m_last, p.q_offset, p.window, p.n[l], first[l], end[l]);
+        if (nl[l] > 0) tile_range(l, m0, m_last, p.q_offset, p.window, nl[l], first[l], end[l]);
         else first[l] = end[l] = 0;
     }
     const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
@@ -168,7 +179,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                         in_mask = (1 << p.page_shift[l]) - 1;
                         for (int bx = 0; bx < n_box; ++bx) {
                             const long long row = (long long)kt * kTileN + bx * rpb;
-                            page[bx] = row < p.n[l] ? tab[row >> p.page_shift[l]] : p.pool_pages[l];
+                            page[bx] = row < nl[l] ? tab[row >> p.page_shift[l]] : p.pool_pages[l];
                         }
                     }
                     if (!mbar_wait(&bar.k_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
@@ -318,14 +329,14 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             if (row_valid) {
                 const float g = p.gate[((long long)b * p.T + t) * 3 + l];
                 bias = g > 0.f ? log2f(g) : -INFINITY;
-                visible_range(l, t + p.q_offset, p.window, p.n[l], 0, lo, hi);
+                visible_range(l, t + p.q_offset, p.window, nl[l], 0, lo, hi);
             }
             // key tiles visible to every row of THIS query tile need no element mask
             int full_first = 0, full_end = 0;
             if (tq0 <= tq1) {
                 long long lo_f, hi_f, lo_l, hi_l;
-                visible_range(l, tq0 + p.q_offset, p.window, p.n[l], 0, lo_f, hi_f);
-                visible_range(l, tq1 + p.q_offset, p.window, p.n[l], 0, lo_l, hi_l);
+                visible_range(l, tq0 + p.q_offset, p.window, nl[l], 0, lo_f, hi_f);
+                visible_range(l, tq1 + p.q_offset, p.window, nl[l], 0, lo_l, hi_l);
                 full_first = (int)((lo_l + kTileN - 1) / kTileN);
                 full_end = (int)(hi_f / kTileN);
                 if (tq1 - tq0 + 1 < kTileM) full_end = full_first;         // ragged query tile: always mask
@@ -467,7 +478,7 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
                 !make_bf16_map(&maps.v[l], P.v, DH, page_rows, fp.H / fp.kv_group, (int)P.pool_pages, P.sn, P.sh, P.sp, rpb))
                 return cudaErrorNotSupported;
             p.table[l] = P.table; p.table_stride[l] = P.table_stride; p.table_head_stride[l] = P.table_head_stride;
-            p.page_shift[l] = P.page_shift; p.box_rows[l] = rpb; p.pool_pages[l] = (int)P.pool_pages;
+            p.page_shift[l] = P.page_shift; p.box_rows[l] = rpb; p.pool_pages[l] = (int)P.pool_pages; p.rows[l] = P.rows;
             continue;
         }
         if (!make_map(&maps.k[l], fp.L[l].k, DH, fp.L[l].n, fp.H / fp.kv_group, fp.B, fp.L[l].sn, fp.L[l].sh, fp.L[l].sb) ||

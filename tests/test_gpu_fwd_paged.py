@@ -49,6 +49,20 @@ def test_paged_forward_matches_oracle(mka, orc, cfg, T, W, q_off):
     assert np.array_equal(np.isfinite(np64(LSE)), live) and np.abs(np64(LSE)[live] - Lr[live]).max() <= 2e-3
 
 
+def test_paged_forward_with_a_length_per_sequence(mka, orc):
+    cfg, T, W = PagedConfig("f_ragged", 58, 3, 4, 2, 128, (400, 400, 150), 16, rows_frac=(1.0, 0.55, 0.0)), 400, 90
+    P, Q, gate = _inputs(cfg, T, cfg.seed)
+    O, LSE = mka.mka_fwd_paged(mka.make_shape(cfg.B, cfg.H, T, cfg.d, 32, W), cfg.H_kv, Q, P["pools_k"], P["pools_v"], P["tables"],
+                               list(cfg.N), gate, rows=P["rows"])
+    Or, Lr = orc.fwd_paged(np64(Q), [np64(k) for k in P["pools_k"]], [np64(v) for v in P["pools_v"]],
+                           [t.cpu().numpy().astype(np.int64) for t in P["tables"]], [r.cpu().numpy() for r in P["rows"]],
+                           cfg.page_rows, np64(gate), W)
+    live = np.isfinite(Lr)                                    # the empty sequence sees nothing: O = 0, LSE = -inf
+    assert live[:2].all() and not live[2].any()
+    check(O, np.where(live[..., None], Or, 0.0), torch.bfloat16, "paged fwd, ragged")
+    assert np.array_equal(np.isfinite(np64(LSE)), live) and np.abs(np64(LSE)[live] - Lr[live]).max() <= 2e-3
+
+
 def test_paged_forward_equals_dense_forward_on_gathered_levels(mka):
     cfg, T, W = PagedConfig("f_same", 56, 2, 4, 2, 128, (512, 512, 128), 16), 512, 200
     P, Q, gate = _inputs(cfg, T, cfg.seed)
