@@ -152,7 +152,69 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     }
     const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
 
-    if (warp == kProducerWarp) {
+    if (warp == kProducerWarp && kPaged) {
+        // Paged levels: the whole warp produces.  Lane i owns box i of every key tile (a box = the rows of one page
+        // that fall into the tile): it looks its page up while the warp waits for the stage to drain and issues its
+        // own copies, so a tile costs one table round trip (overlapped) and four warp-wide copy instructions.
+        if (lane == 0) {
+            mbar_expect_tx(&bar.q_full, kNumQ * C::kTileBytes);
+#pragma unroll
+            for (int q = 0; q < kNumQ; ++q)
+#pragma unroll
+                for (int pn = 0; pn < C::kPanels; ++pn)
+                    tma_load_4d(sQ + q * C::kTileBytes + pn * kPanelBytes, &maps.q, pn * 64, (int)(m0 + q * kTileM), h, b, &bar.q_full);
+        }
+        int issued = 0;
+        bool ok = true;
+        const int kvh = h / p.kv_group;
+        for (int l = 0; l < 3 && ok; ++l) {
+            if (first[l] >= end[l]) continue;
+            const int* tab = p.table[l] + (long long)b * p.table_stride[l] + (long long)kvh * p.table_head_stride[l];
+            const int rpb = p.box_rows[l];
+            const bool mine = lane < kTileN / rpb;
+            const int in_mask = (1 << p.page_shift[l]) - 1;
+            for (int kt = first[l]; kt < end[l]; ++kt) {
+                const int s = issued % C::kStages;
+                const uint32_t ph = (uint32_t)(issued / C::kStages) & 1u;
+                // a box past the level's last row is aimed past the pool, where the copy engine fills zeros as it does
+                // past a dense level's end
+                const long long row = (long long)kt * kTileN + lane * rpb;
+                int page = p.pool_pages[l];
+                if (mine && row < nl[l]) page = tab[row >> p.page_shift[l]];
+                const int in_row = (int)(row & in_mask);
+                if (!mbar_wait_warp(&bar.k_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
+                if (lane == 0) mbar_expect_tx(&bar.k_full[s], C::kTileBytes);
+                __syncwarp();
+                if (mine) {
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes + lane * rpb * 128, &maps.k[l], pn * 64, in_row, kvh, page,
+                                    &bar.k_full[s]);
+                }
+                if (!mbar_wait_warp(&bar.v_empty[s], ph ^ 1u, abortp)) {           // gave up with this stage's K copies in flight
+                    mbar_wait_warp(&bar.k_full[s], ph, abortp);
+                    ok = false;
+                    break;
+                }
+                if (lane == 0) mbar_expect_tx(&bar.v_full[s], C::kTileBytes);
+                __syncwarp();
+                if (mine) {
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes + lane * rpb * 128, &maps.v[l], pn * 64, in_row, kvh, page,
+                                    &bar.v_full[s]);
+                }
+                ++issued;
+            }
+        }
+        // Before leaving, make sure every copy issued has landed (bounded): the shared memory must not be handed to
+        // another CTA with a bulk copy still in flight.  (A stage whose wait failed got no copies.)
+        mbar_wait_warp(&bar.q_full, 0, abortp);
+        for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i) {
+            mbar_wait_warp(&bar.k_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+            mbar_wait_warp(&bar.v_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+        }
+    } else if (warp == kProducerWarp) {
         if (lane == 0) {
             mbar_expect_tx(&bar.q_full, kNumQ * C::kTileBytes);
 #pragma unroll
@@ -164,51 +226,21 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             bool ok = true;
             const int kvh = h / p.kv_group;
             for (int l = 0; l < 3 && ok; ++l) {
-                const int* tab = kPaged ? p.table[l] + (long long)b * p.table_stride[l] + (long long)kvh * p.table_head_stride[l] : nullptr;
                 for (int kt = first[l]; kt < end[l]; ++kt) {
                     const int e = issued_k;
                     const int s = e % C::kStages;
                     const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
-                    // paged: the pool page of every box of this tile (K and V share them); a box past the level's last
-                    // row is aimed past the pool, where the copy engine fills zeros as it does past a dense level's end
-                    int page[16];
-                    int n_box = 0, rpb = kTileN, in_mask = 0;
-                    if (kPaged) {
-                        rpb = p.box_rows[l];
-                        n_box = kTileN / rpb;
-                        in_mask = (1 << p.page_shift[l]) - 1;
-                        for (int bx = 0; bx < n_box; ++bx) {
-                            const long long row = (long long)kt * kTileN + bx * rpb;
-                            page[bx] = row < nl[l] ? tab[row >> p.page_shift[l]] : p.pool_pages[l];
-                        }
-                    }
                     if (!mbar_wait(&bar.k_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(&bar.k_full[s], C::kTileBytes);
-                    if (!kPaged) {
 #pragma unroll
-                        for (int pn = 0; pn < C::kPanels; ++pn)
-                            tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes, &maps.k[l], pn * 64, kt * kTileN, kvh, b, &bar.k_full[s]);
-                    } else {
-                        for (int bx = 0; bx < n_box; ++bx)
-#pragma unroll
-                            for (int pn = 0; pn < C::kPanels; ++pn)
-                                tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes + bx * rpb * 128, &maps.k[l], pn * 64,
-                                            (kt * kTileN + bx * rpb) & in_mask, kvh, page[bx], &bar.k_full[s]);
-                    }
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sK + s * C::kTileBytes + pn * kPanelBytes, &maps.k[l], pn * 64, kt * kTileN, kvh, b, &bar.k_full[s]);
                     ++issued_k;
                     if (!mbar_wait(&bar.v_empty[s], ph ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(&bar.v_full[s], C::kTileBytes);
-                    if (!kPaged) {
 #pragma unroll
-                        for (int pn = 0; pn < C::kPanels; ++pn)
-                            tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes, &maps.v[l], pn * 64, kt * kTileN, kvh, b, &bar.v_full[s]);
-                    } else {
-                        for (int bx = 0; bx < n_box; ++bx)
-#pragma unroll
-                            for (int pn = 0; pn < C::kPanels; ++pn)
-                                tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes + bx * rpb * 128, &maps.v[l], pn * 64,
-                                            (kt * kTileN + bx * rpb) & in_mask, kvh, page[bx], &bar.v_full[s]);
-                    }
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sV + s * C::kTileBytes + pn * kPanelBytes, &maps.v[l], pn * 64, kt * kTileN, kvh, b, &bar.v_full[s]);
                     ++issued_v;
                 }
             }
