@@ -271,6 +271,18 @@ mka_status mka_bwd(const mka_shape* shape, const void* Q, const mka_level L[3], 
 mka_status mka_fuse_kv(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype, const mka_level L[3],
                        const float* gate, const mka_level_grad* dst, int64_t dst_offset, void* stream);
 
+/*
+ * mka_fuse_kv with a PAGED destination: the fused rows of sequence b are appended to a paged cache at logical rows
+ * dst_offset + dst_offsets[b] + j (dst_offsets: device int32 [B], or NULL = 0 for all), found through dst->page_table
+ * as in mka_paged_level (one table per sequence; table_head_stride is ignored).  dst->k, dst->v are WRITTEN although
+ * the struct declares them const; H counts the heads of the pool.  dst->n and the table must cover dst_offset + n rows
+ * plus the largest per-sequence offset (the latter is the caller's promise: it lives on the device).  Everything else
+ * as mka_fuse_kv.
+ */
+mka_status mka_fuse_kv_paged(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype, const mka_level L[3],
+                             const float* gate, const mka_paged_level* dst, int64_t dst_offset, const int32_t* dst_offsets,
+                             void* stream);
+
 /* Causal summaries of mka_l2_summary. */
 typedef enum { MKA_SUMMARY_MEAN = 0, MKA_SUMMARY_EMA = 1 } mka_summary;
 

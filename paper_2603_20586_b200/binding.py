@@ -26,7 +26,7 @@ TILE = 128
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
            "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_l2_summary_workspace_bytes", "mka_l2_summary_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes",
-           "mka_decode_paged", "mka_decode_paged_workspace_bytes", "mka_l3_index", "mka_l3_retrieve", "mka_fwd_paged"]
+           "mka_decode_paged", "mka_decode_paged_workspace_bytes", "mka_l3_index", "mka_l3_retrieve", "mka_fwd_paged", "mka_fuse_kv_paged"]
 
 
 class MkaError(RuntimeError):
@@ -99,6 +99,8 @@ def _load() -> ctypes.CDLL:
     lib.mka_decode_paged.argtypes = [ctypes.POINTER(mka_shape), i32, vp, ctypes.POINTER(mka_paged_level), vp, vp, vp, vp,
                                      ctypes.c_size_t, vp]
     lib.mka_fwd_paged.argtypes = lib.mka_decode_paged.argtypes
+    lib.mka_fuse_kv_paged.argtypes = [i32, i32, i64, i32, i32, ctypes.POINTER(mka_level), vp, ctypes.POINTER(mka_paged_level), i64,
+                                      vp, vp]
     lib.mka_l3_index.argtypes = [vp, i64, i32, i32, i32, i64, i64, i64, vp, i32, vp, vp]
     lib.mka_l3_retrieve.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.mka_l2_summary_kernel_kind.argtypes = [i32, i64, i32, i32, ctypes.c_size_t]
@@ -244,6 +246,23 @@ def _paged_levels(pools_k, pools_v, tables, rows, n):
                                  tab.stride(1) if tab.dim() == 3 else 0, k.shape[2], k.stride(0), k.stride(1), k.stride(2),
                                  k.shape[0])
     return arr
+
+
+def mka_fuse_kv_paged(K, V, gate, pool_k, pool_v, table, dst_offset=0, dst_offsets=None, stream=None):
+    """Route-fusion of token-aligned levels K[l], V[l] ([B, H, n, d] or None) with gate [B, n, 3], appended to the paged
+    cache pool_k / pool_v [pages, H, page_rows, d] through table int32 [B, pages] at logical rows dst_offset
+    (+ dst_offsets[b]) + j."""
+    ref = next(k for k in K if k is not None)
+    B, H, n, d = ref.shape
+    assert gate.is_contiguous() and gate.dtype == torch.float32 and tuple(gate.shape) == (B, n, 3)
+    assert pool_k.dim() == 4 and pool_k.stride(3) == 1 and pool_v.stride() == pool_k.stride() and pool_k.dtype == ref.dtype
+    assert table.dtype == torch.int32 and table.dim() == 2 and table.stride(1) == 1
+    assert dst_offsets is None or (dst_offsets.dtype == torch.int32 and dst_offsets.is_contiguous())
+    dst = mka_paged_level(pool_k.data_ptr(), pool_v.data_ptr(), table.data_ptr(), None, table.shape[1] * pool_k.shape[2],
+                          table.stride(0), 0, pool_k.shape[2], pool_k.stride(0), pool_k.stride(1), pool_k.stride(2), pool_k.shape[0])
+    _check(lib.mka_fuse_kv_paged(B, H, n, d, _dt(ref), _levels(K, V), _ptr(gate), ctypes.byref(dst), dst_offset, _ptr(dst_offsets),
+                                 _stream(stream)), "mka_fuse_kv_paged")
+    return pool_k, pool_v
 
 
 def mka_fwd_paged(shape: mka_shape, H_kv: int, Q, pools_k, pools_v, tables, n, gate, rows=None, O=None, LSE=None, ws=None,

@@ -512,6 +512,46 @@ int32_t mka_l2_summary_kernel_kind(int32_t B, int64_t T, int32_t D, int32_t dtyp
     return T >= 512 && narrow && ws_bytes >= kWsHeader + l2_summary_seg_workspace(B, T, D, dtype) ? 1 : 0;
 }
 
+mka_status mka_fuse_kv_paged(int32_t B, int32_t H, int64_t n, int32_t d, int32_t dtype, const mka_level L[3],
+                             const float* gate, const mka_paged_level* dst, int64_t dst_offset, const int32_t* dst_offsets,
+                             void* stream) {
+    if (dtype != MKA_BF16 && dtype != MKA_F32) return MKA_ERR_ARG;
+    if (!L || !dst) return MKA_ERR_ARG;
+    if (B < 0 || H < 0 || n < 0 || dst_offset < 0) return MKA_ERR_SHAPE;
+    const int elems = dtype == MKA_BF16 ? 8 : 4;
+    if (d <= 0 || d > 1024 || d % elems) return MKA_ERR_SHAPE;
+    const int pr = dst->page_rows;
+    if (pr <= 0 || (pr & (pr - 1)) != 0) return MKA_ERR_SHAPE;
+    if (dst->table_stride * pr < dst_offset + n || dst->n < dst_offset + n) return MKA_ERR_SHAPE;   // without the per-sequence offsets
+    if (B == 0 || H == 0 || n == 0) return MKA_OK;
+    if (!gate || !dst->k || !dst->v || !dst->page_table) return MKA_ERR_ARG;
+    if (dst->stride_n < d || dst->stride_page < 0 || dst->stride_h < 0) return MKA_ERR_SHAPE;
+    if (!aligned16(dst->k) || !aligned16(dst->v) || dst->stride_n % elems || dst->stride_page % elems || dst->stride_h % elems)
+        return MKA_ERR_ALIGN;
+    int present = 0;
+    LevelDev lv[3];
+    for (int l = 0; l < 3; ++l) {
+        if (L[l].n != 0 && L[l].n != n) return MKA_ERR_SHAPE;
+        lv[l].k = L[l].k; lv[l].v = L[l].v; lv[l].n = L[l].n;
+        lv[l].sb = L[l].stride_b; lv[l].sh = L[l].stride_h; lv[l].sn = L[l].stride_n;
+        if (L[l].n == 0) continue;
+        ++present;
+        if (!L[l].k || !L[l].v) return MKA_ERR_ARG;
+        if (L[l].stride_n < d || L[l].stride_b < 0 || L[l].stride_h < 0) return MKA_ERR_SHAPE;
+        if (!aligned16(L[l].k) || !aligned16(L[l].v) || L[l].stride_n % elems || L[l].stride_b % elems || L[l].stride_h % elems)
+            return MKA_ERR_ALIGN;
+    }
+    if (!present) return MKA_ERR_ARG;
+    LevelGradDev out;
+    out.dk = const_cast<void*>(dst->k); out.dv = const_cast<void*>(dst->v); out.n = dst->n;
+    out.sb = dst->stride_page; out.sh = dst->stride_h; out.sn = dst->stride_n;
+    int shift = 0;
+    while ((1 << shift) < pr) ++shift;
+    cudaError_t e = launch_fuse_kv(lv, out, gate, B, H, n, d, dst_offset, dtype, static_cast<cudaStream_t>(stream),
+                                   dst->page_table, dst->table_stride, shift, dst_offsets);
+    return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+}
+
 mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_t dtype, int32_t kind, float beta, float* state,
                           int64_t n_prev, void* M2, void* ws, size_t ws_bytes, void* stream) {
     if (dtype != MKA_BF16 && dtype != MKA_F32) return MKA_ERR_ARG;

@@ -153,7 +153,8 @@ cudaError_t launch_router_bwd(const void* R, int r_dtype, const float* dG, long 
                               float* db_r, float* partial, int n_row_chunks, cudaStream_t st);
 
 cudaError_t launch_fuse_kv(const LevelDev L[3], const LevelGradDev& out, const float* gate, int B, int H, long long n, int d,
-                           long long dst_offset, int dtype, cudaStream_t st);
+                           long long dst_offset, int dtype, cudaStream_t st, const int* dst_table = nullptr,
+                           long long dst_table_stride = 0, int dst_page_shift = 0, const int* dst_offsets = nullptr);
 cudaError_t launch_l2_summary(const void* X, void* M2, float* state, int use_state, long long n_prev, int B, long long T, int D,
                               int dtype, int kind, float beta, unsigned int* status, cudaStream_t st);
 size_t l2_summary_seg_workspace(int B, long long T, int D, int dtype);

@@ -54,6 +54,12 @@ struct FuseParams {
     const float* gate;    // [B, n, 3]
     long long n, dst_offset;
     int B, H, d;
+    // paged destination (dst_table != null): out.sb is then the stride between PAGES and row r of sequence b lives
+    // in page dst_table[b * dst_table_stride + r / page_rows]
+    const int* dst_table;
+    const int* dst_offsets;      // per-sequence offset added to dst_offset, or null
+    long long dst_table_stride;
+    int dst_page_shift;
 };
 
 template <typename T>
@@ -88,7 +94,14 @@ __global__ void __launch_bounds__(256) fuse_kv_kernel(const FuseParams p, const 
                 Vec<T>::acc(vv[l], w[l], av);
             }
         }
-        const long long oo = b * p.out.sb + h * p.out.sh + (p.dst_offset + j) * p.out.sn + c;
+        long long oo;
+        if (p.dst_table) {
+            const long long r = p.dst_offset + (p.dst_offsets ? p.dst_offsets[b] : 0) + j;
+            const long long page = p.dst_table[b * p.dst_table_stride + (r >> p.dst_page_shift)];
+            oo = page * p.out.sb + h * p.out.sh + (r & ((1LL << p.dst_page_shift) - 1)) * p.out.sn + c;
+        } else {
+            oo = b * p.out.sb + h * p.out.sh + (p.dst_offset + j) * p.out.sn + c;
+        }
         *reinterpret_cast<uint4*>(static_cast<T*>(p.out.dk) + oo) = Vec<T>::pack(ak);
         *reinterpret_cast<uint4*>(static_cast<T*>(p.out.dv) + oo) = Vec<T>::pack(av);
     }
@@ -97,10 +110,12 @@ __global__ void __launch_bounds__(256) fuse_kv_kernel(const FuseParams p, const 
 }  // namespace
 
 cudaError_t launch_fuse_kv(const LevelDev L[3], const LevelGradDev& out, const float* gate, int B, int H, long long n, int d,
-                           long long dst_offset, int dtype, cudaStream_t st) {
+                           long long dst_offset, int dtype, cudaStream_t st, const int* dst_table, long long dst_table_stride,
+                           int dst_page_shift, const int* dst_offsets) {
     FuseParams p;
     for (int l = 0; l < 3; ++l) p.L[l] = L[l];
     p.out = out; p.gate = gate; p.n = n; p.dst_offset = dst_offset; p.B = B; p.H = H; p.d = d;
+    p.dst_table = dst_table; p.dst_table_stride = dst_table_stride; p.dst_page_shift = dst_page_shift; p.dst_offsets = dst_offsets;
     const int elems = dtype == MKA_BF16 ? 8 : 4;
     const long long total = (long long)B * H * n * (d / elems);
     if (total == 0) return cudaSuccess;

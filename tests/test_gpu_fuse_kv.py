@@ -97,3 +97,34 @@ def test_fuse_kv_rejects_bad_arguments(mka):
     with pytest.raises(mka.MkaError) as e:
         mka.mka_fuse_kv([K[0], K[1][:, :, :8], K[2]], [V[0], V[1][:, :, :8], V[2]], gate)   # levels not token-aligned
     assert e.value.code == 2
+
+
+def test_fuse_kv_into_a_paged_cache(mka, orc):
+    """The fused rows land where the page table says, at a different offset per sequence; nothing else is touched."""
+    B, H, n, d, pr = 3, 4, 50, 64, 16
+    Ks = [approx_normal(71, 10 + l, 0, B * H * n * d, 1.0, "cpu", torch.bfloat16).view(B, H, n, d).cuda() for l in range(3)]
+    Vs = [approx_normal(71, 20 + l, 0, B * H * n * d, 1.0, "cpu", torch.bfloat16).view(B, H, n, d).cuda() for l in range(3)]
+    gate = torch.softmax(approx_normal(71, 30, 0, B * n * 3, 1.0, "cpu", torch.float32).view(B, n, 3), -1).cuda().contiguous()
+    pages_per_seq = 8                                             # room for 128 rows per sequence
+    gen = torch.Generator().manual_seed(71)
+    table = torch.randperm(B * pages_per_seq + 2, generator=gen)[:B * pages_per_seq].int().view(B, pages_per_seq).cuda()
+    pool_k = torch.full((B * pages_per_seq + 2, H, pr, d), 7.0, dtype=torch.bfloat16, device="cuda")
+    pool_v = torch.full_like(pool_k, -7.0)
+    offs = torch.tensor([0, 13, 40], dtype=torch.int32, device="cuda")
+    base = 5
+    mka.mka_fuse_kv_paged(Ks, Vs, gate, pool_k, pool_v, table, dst_offset=base, dst_offsets=offs)
+    rk = orc.route_fuse(Ks, np64(gate))                           # [B, H, n, d]
+    rv = orc.route_fuse(Vs, np64(gate))
+    dense_k = pool_k[table.long()].permute(0, 2, 1, 3, 4).reshape(B, H, pages_per_seq * pr, d)
+    dense_v = pool_v[table.long()].permute(0, 2, 1, 3, 4).reshape(B, H, pages_per_seq * pr, d)
+    for b in range(B):
+        o = base + int(offs[b])
+        ek = np.abs(np64(dense_k[b, :, o:o + n]) - rk[b])
+        ev = np.abs(np64(dense_v[b, :, o:o + n]) - rv[b])
+        assert ek.max() <= BF16_MAX and ev.max() <= BF16_MAX and ek.mean() <= BF16_MEAN and ev.mean() <= BF16_MEAN
+        untouched = torch.ones(pages_per_seq * pr, dtype=torch.bool, device="cuda")
+        untouched[o:o + n] = False
+        assert (dense_k[b][:, untouched] == 7.0).all() and (dense_v[b][:, untouched] == -7.0).all()
+    used = torch.zeros(pool_k.shape[0], dtype=torch.bool, device="cuda")
+    used[table.flatten().long()] = True
+    assert (pool_k[~used] == 7.0).all()                           # pages that belong to nobody
