@@ -98,8 +98,8 @@ typedef struct mka_shape {
     int32_t kv_heads; /* grouped-query sharing (the paper evaluates on GQA models): 0 or H = one KV head per query
                          head; otherwise H % kv_heads == 0, the levels hold kv_heads heads ([B, kv_heads, n, d]) and
                          query head h reads KV head h / (H / kv_heads).  Honoured by mka_fwd, mka_decode and
-                         the tensor-core path of mka_bwd (dK, dV then hold kv_heads heads, summed over each group;
-                         the CUDA-core backward returns MKA_ERR_UNSUPPORTED); the paged decode has its own H_kv */
+                         mka_bwd (dK, dV then hold kv_heads heads, summed over each group); the paged entry points
+                         take H_kv as an argument instead */
 } mka_shape;
 
 /* Split table of the decode kernel: level l is cut into n_chunks[l] chunks of chunk_rows rows (the last

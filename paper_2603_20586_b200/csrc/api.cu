@@ -447,7 +447,6 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
     p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s); p.kv_group = kv_group_of(s);
     const bool tc = !(s->flags & MKA_FLAG_FORCE_SIMT) && bwd_tc_eligible(p, s->dtype);
-    if (!tc && p.kv_group != 1) return MKA_ERR_UNSUPPORTED;   // shared KV heads: only the tensor-core kernels sum over a group
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
     cudaError_t e;

@@ -66,8 +66,8 @@ __global__ void __launch_bounds__(kThreads) bwd_dq_kernel(const BwdParams p) {
         visible_range(lvl, t0 + p.q_offset, p.window, L.n, 0, lo_f, hi_f);
         visible_range(lvl, t_last + p.q_offset, p.window, L.n, 0, lo_l, hi_l);
         const long long lo = lo_f, hi = hi_l > hi_f ? hi_l : hi_f;
-        const T* Kp = static_cast<const T*>(L.k) + b * L.sb + h * L.sh;
-        const T* Vp = static_cast<const T*>(L.v) + b * L.sb + h * L.sh;
+        const T* Kp = static_cast<const T*>(L.k) + b * L.sb + (h / p.kv_group) * L.sh;
+        const T* Vp = static_cast<const T*>(L.v) + b * L.sb + (h / p.kv_group) * L.sh;
         float lam[kWarpRows];
         long long rlo[kWarpRows], rhi[kWarpRows];
 #pragma unroll
@@ -165,15 +165,12 @@ __global__ void __launch_bounds__(kThreads) bwd_dkv_kernel(const BwdParams p, co
     float* gs = qs + kRows * LD;      // [kRows][LD]  dO tile
     __shared__ float s_lse[kRows], s_dlt[kRows], s_lam[kRows];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int b = blockIdx.z, h = blockIdx.y;
-    const long long bh = (long long)b * p.H + h;
+    const int b = blockIdx.z, h = blockIdx.y;               // h: KV head; its query heads h * G .. h * G + G - 1 are summed
     const LevelDev L = p.L[lvl];
     const LevelGradDev dL = p.dL[lvl];
     const long long j0 = (long long)blockIdx.x * kKeys;
     const T* Kp = static_cast<const T*>(L.k) + b * L.sb + h * L.sh;
     const T* Vp = static_cast<const T*>(L.v) + b * L.sb + h * L.sh;
-    const T* Q = static_cast<const T*>(p.Q) + bh * p.T * DH;
-    const T* dO = static_cast<const T*>(p.dO) + bh * p.T * DH;
     for (int i = threadIdx.x; i < kKeys * DH; i += kThreads) {
         long long j = j0 + i / DH;
         ksm[i] = j < L.n ? Elem<T>::ld(Kp + j * L.sn + (i % DH)) * p.scale : 0.f;
@@ -192,6 +189,10 @@ __global__ void __launch_bounds__(kThreads) bwd_dkv_kernel(const BwdParams p, co
     else if (lvl == 1) { t_lo = j0 - p.q_offset; }
     if (t_lo < 0) t_lo = 0;
     if (t_hi > p.T) t_hi = p.T;
+    for (int gq = 0; gq < p.kv_group; ++gq) {
+    const long long bh = (long long)b * p.H + (long long)h * p.kv_group + gq;
+    const T* Q = static_cast<const T*>(p.Q) + bh * p.T * DH;
+    const T* dO = static_cast<const T*>(p.dO) + bh * p.T * DH;
     for (long long tt = (t_lo / kRows) * kRows; tt < t_hi; tt += kRows) {
         __syncthreads();
         for (int i = threadIdx.x; i < kRows * DH; i += kThreads) {
@@ -259,6 +260,7 @@ __global__ void __launch_bounds__(kThreads) bwd_dkv_kernel(const BwdParams p, co
             }
         }
     }
+    }   // query heads of the group
     T* dKp = static_cast<T*>(dL.dk) + b * dL.sb + h * dL.sh;
     T* dVp = static_cast<T*>(dL.dv) + b * dL.sb + h * dL.sh;
 #pragma unroll
@@ -316,7 +318,7 @@ cudaError_t launch_t(const BwdParams& p, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         for (int lvl = 0; lvl < 3; ++lvl) {
             if (p.L[lvl].n == 0) continue;
-            dim3 grid((unsigned)((p.L[lvl].n + kKeys - 1) / kKeys), p.H, p.B);
+            dim3 grid((unsigned)((p.L[lvl].n + kKeys - 1) / kKeys), p.H / (p.kv_group > 0 ? p.kv_group : 1), p.B);
             bwd_dkv_kernel<T, DH><<<grid, kThreads, smem, st>>>(p, lvl);
             if ((e = cudaGetLastError()) != cudaSuccess) return e;
         }

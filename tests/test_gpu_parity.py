@@ -354,14 +354,10 @@ def test_grouped_query_heads_argument_checks(mka):
         mka.mka_fwd(mka.make_shape(B, H, T, d, 64, 32, kv_heads=4), Q, P["K"], P["V"], gate)
     assert e.value.code == 2
     O, LSE = mka.mka_fwd(mka.make_shape(B, H, T, d, 64, 32, kv_heads=2), Q, P["K"], P["V"], gate)
-    with pytest.raises(mka.MkaError) as e:                       # the CUDA-core backward does not sum over a group
-        mka.mka_bwd(mka.make_shape(B, H, T, d, 64, 32, flags=1, kv_heads=2), Q, P["K"], P["V"], gate, O, LSE,
-                    torch.zeros_like(Q), want_router_grad=False)
-    assert e.value.code == 5
 
 
-@pytest.mark.parametrize("d", [128, 64])
-def test_bwd_with_grouped_query_heads(mka, orc, d):
+@pytest.mark.parametrize("d,flags", [(128, 0), (64, 0), (64, 1)])
+def test_bwd_with_grouped_query_heads(mka, orc, d, flags):
     """dK, dV of a shared KV head are the sums over the query heads of its group; dQ, dG as for the repeated heads."""
     B, H, H_kv, T, W, N = 2, 6, 2, 260, 70, (260, 260, 40)
     G = H // H_kv
@@ -369,8 +365,8 @@ def test_bwd_with_grouped_query_heads(mka, orc, d):
     Q = approx_normal(43, 50, 0, B * H * T * d, 1.0, "cpu", torch.bfloat16).view(B, H, T, d).cuda()
     dO = approx_normal(43, 51, 0, B * H * T * d, 1.0, "cpu", torch.bfloat16).view(B, H, T, d).cuda()
     gate = mka.mka_router(P["X"], P["W_r"], None)
-    shape = mka.make_shape(B, H, T, d, 64, W, kv_heads=H_kv)
-    assert mka.mka_bwd_kernel_kind(shape, P["K"], P["V"]) == 1
+    shape = mka.make_shape(B, H, T, d, 64, W, flags=flags, kv_heads=H_kv)
+    assert mka.mka_bwd_kernel_kind(shape, P["K"], P["V"]) == (0 if flags else 1)
     O, LSE = mka.mka_fwd(shape, Q, P["K"], P["V"], gate)
     g = mka.mka_bwd(shape, Q, P["K"], P["V"], gate, O, LSE, dO, R=P["X"])
     Kr = [np.repeat(np64(k), G, axis=1) for k in P["K"]]
