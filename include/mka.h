@@ -157,6 +157,8 @@ mka_status mka_fwd(const mka_shape* shape, const void* Q, const mka_level L[3], 
  * (window and q_offset are ignored).  Each chunk of the split table produces an un-gated partial
  * (max, sum, accumulator); a second kernel combines them with the gate in log-sum-exp form.
  *   q [B, H, d];  gate [B, 3] f32;  O [B, H, d];  LSE [B, H] f32 or NULL.
+ * With shape->kv_heads < H (at most 16 query heads per KV head) the grouped-query kernel of mka_decode_paged runs on the
+ * dense levels and reads every cached row once per KV head; ask mka_workspace_bytes with the same shape.
  */
 mka_status mka_decode(const mka_shape* shape, const void* q, const mka_level L[3], const float* gate,
                       void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);

@@ -127,12 +127,23 @@ mka_status mka_fwd_tile_range(const mka_shape* s, const int64_t n_level[3], int3
     return MKA_OK;
 }
 
+static mka_status paged_plan(const int64_t n_level[3], int32_t B, int32_t H_kv, mka_decode_plan_t* plan);
+
+// Grouped heads in the dense decode run the grouped-query kernel (every cached row read once per KV head).
+static bool decode_uses_grouped_kernel(const mka_shape* s) {
+    return s->kv_heads > 0 && s->kv_heads < s->H && s->H % s->kv_heads == 0 && s->H / s->kv_heads <= 16;
+}
+
 size_t mka_workspace_bytes(const mka_shape* s, const int64_t n_level[3], int32_t which) {
     if (!s || !n_level) return 0;
     if (which == MKA_WS_FWD) return kWsHeader;
     if (which == MKA_WS_DECODE) {
         mka_decode_plan_t plan;
-        if (mka_decode_plan(n_level, s->B, s->H, s->d, &plan) != MKA_OK) return 0;
+        if (decode_uses_grouped_kernel(s)) {
+            if (paged_plan(n_level, s->B, s->kv_heads, &plan) != MKA_OK) return 0;
+        } else if (mka_decode_plan(n_level, s->B, s->H, s->d, &plan) != MKA_OK) {
+            return 0;
+        }
         return kWsHeader + round_up((size_t)s->B * s->H * plan.total_chunks * (s->d + 2) * sizeof(float), 256);
     }
     if (which == MKA_WS_BWD) {
@@ -205,6 +216,34 @@ mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], c
     int64_t n_level[3] = {L[0].n, L[1].n, L[2].n};
     size_t need = mka_workspace_bytes(s, n_level, MKA_WS_DECODE);
     if (!ws || ws_bytes < need) return MKA_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (decode_uses_grouped_kernel(s)) {
+        // dense levels seen as paged ones with a single page per sequence (no table: the page is the batch index)
+        mka_decode_plan_t plan;
+        paged_plan(n_level, s->B, s->kv_heads, &plan);
+        if ((long long)s->B * s->H * plan.total_chunks > 0x7fffffffLL) return MKA_ERR_SHAPE;
+        DecodePagedParams pp;
+        memset(&pp, 0, sizeof(pp));
+        for (int l = 0; l < 3; ++l) {
+            pp.L[l].k = L[l].k; pp.L[l].v = L[l].v; pp.L[l].table = nullptr; pp.L[l].rows = nullptr; pp.L[l].n = L[l].n;
+            pp.L[l].sp = L[l].stride_b; pp.L[l].sh = L[l].stride_h; pp.L[l].sn = L[l].stride_n;
+            pp.L[l].page_shift = 40;
+            pp.n_chunks[l] = plan.n_chunks[l];
+        }
+        pp.q = q; pp.gate = gate; pp.B = s->B; pp.H = s->H; pp.H_kv = s->kv_heads; pp.d = s->d; pp.scale = resolve_scale(s);
+        pp.chunk_rows = plan.chunk_rows; pp.total_chunks = plan.total_chunks;
+        pp.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeader);
+        DecodeParams c;
+        memset(&c, 0, sizeof(c));
+        c.O = O; c.LSE = LSE; c.gate = gate; c.B = s->B; c.H = s->H; c.d = s->d;
+        c.total_chunks = plan.total_chunks; c.partial = pp.partial;
+        for (int l = 0; l < 3; ++l) c.n_chunks[l] = plan.n_chunks[l];
+        if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
+        cudaError_t e = launch_decode_paged(pp, cs);
+        if (e == cudaSuccess) e = launch_decode_combine(c, cs);
+        if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;
+        return e == cudaSuccess ? MKA_OK : MKA_ERR_CUDA;
+    }
     mka_decode_plan_t plan;
     mka_decode_plan(n_level, s->B, s->H, s->d, &plan);
     if ((long long)s->B * s->H * plan.total_chunks > 0x7fffffffLL) return MKA_ERR_SHAPE;
@@ -217,7 +256,6 @@ mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], c
     for (int l = 0; l < 3; ++l) p.n_chunks[l] = plan.n_chunks[l];
     p.total_chunks = plan.total_chunks;
     p.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeader);
-    cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
     cudaError_t e = launch_decode(p, cs);
     if (e == cudaErrorNotSupported) return MKA_ERR_UNSUPPORTED;

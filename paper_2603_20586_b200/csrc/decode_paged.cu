@@ -102,11 +102,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_paged_kernel(const DecodeP
     // this chunk's slice of the page table, fetched once: at most one entry per row of the chunk
     __shared__ int s_pages[kSliceCap];
     const long long page0 = r_begin >> shift;
-    const int* table = L.table + (long long)b * L.table_stride + (long long)kvh * L.table_head_stride + page0;
+    // (a dense level comes without a table: it is one page per sequence, the page being the batch index)
+    const int* table = L.table ? L.table + (long long)b * L.table_stride + (long long)kvh * L.table_head_stride + page0 : nullptr;
     const long long n_pages = ((r_end - 1) >> shift) - page0 + 1;
     const bool sliced = n_pages <= kSliceCap;              // (tiny pages in a long chunk: look the table up in place)
     if (sliced)
-        for (int i = tid; i < (int)n_pages; i += kThreads) s_pages[i] = table[i];
+        for (int i = tid; i < (int)n_pages; i += kThreads) s_pages[i] = table ? table[i] : b;
     __syncthreads();
     const __nv_bfloat16* Kbase = static_cast<const __nv_bfloat16*>(L.k) + (long long)kvh * L.sh;
     const __nv_bfloat16* Vbase = static_cast<const __nv_bfloat16*>(L.v) + (long long)kvh * L.sh;

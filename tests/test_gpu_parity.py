@@ -380,3 +380,16 @@ def test_bwd_with_grouped_query_heads(mka, orc, d, flags):
         check(g["dK"][l], dk, torch.bfloat16, f"grouped-query dK{l}")
         check(g["dV"][l], dv, torch.bfloat16, f"grouped-query dV{l}")
     assert np.abs(np64(g["dG"]) - ref["dG"]).max() <= 2e-2
+
+
+def test_decode_with_more_than_16_heads_per_group_takes_the_plain_kernel(mka, orc):
+    """17 query heads on one KV head: beyond the grouped-query kernel's 16 rows, so the plain kernel reads the KV head per head."""
+    B, H, d, N = 1, 17, 64, (40, 300, 64)
+    P = problem(44, B, 1, 1, d, N, 64, torch.bfloat16)
+    q = approx_normal(44, 50, 0, B * H * d, 1.0, "cpu", torch.bfloat16).view(B, H, d).cuda()
+    gate = torch.tensor([[0.2, 0.5, 0.3]], device="cuda")
+    O, _ = mka.mka_decode(mka.make_shape(B, H, 1, d, 64, kv_heads=1), q, P["K"], P["V"], gate)
+    Kr = [np.repeat(np64(k), H, axis=1) for k in P["K"]]
+    Vr = [np.repeat(np64(v), H, axis=1) for v in P["V"]]
+    Or, _ = orc.fwd(np64(q)[:, :, None], Kr, Vr, np64(gate)[:, None], 1, decode=True)
+    check(O.view(B, H, 1, d), Or, torch.bfloat16, "decode, 17 heads on one KV head")
