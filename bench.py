@@ -58,7 +58,7 @@ NCU_TRAFFIC = {
     "bwd_dq_tc_kernel@c5": (220.282624e6 + 29.623808e6, 1 * 16),
     "l2_summary_seg_kernel@s3": (100.972800e6 + 55.965184e6, 12288.0 / 32768.0),   # captured on 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8),
-    "decode_paged_kernel@g4": (293.680640e6 + 3.976448e6, 1 * 4),   # captured on one of the four sequences (g4p)
+    "decode_paged_kernel@g4": (293.713664e6 + 3.592192e6, 1 * 4),   # captured on one of the four sequences (g4p)
     "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1),            # captured on one of the four sequences (r3p)
     "bwd_dkv_tc_kernel@c5": (220.432640e6 + 115.097856e6, 1 * 16),
 }
