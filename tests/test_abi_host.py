@@ -110,3 +110,59 @@ def test_forward_tile_ranges_match_mask_enumeration(mka, T, W, q_off, N):
             full = [kt for kt in range(first, end)
                     if all(set(range(kt * 128, kt * 128 + 128)) <= v for v in vis)]
             assert full == list(range(ff, fe)), (q_tile, level, full, ff, fe)
+
+
+def test_widened_entry_points_validate_on_the_host(mka):
+    """Paged, grouped-head, summary and recall entry points reject bad arguments before anything is launched."""
+    b = mka.binding
+    pl = (b.mka_paged_level * 3)()
+    dec = mka.make_shape(1, 8, 1, 128)
+    assert mka.lib.mka_decode_paged(ctypes.byref(dec), 3, None, pl, None, None, None, None, 0, None) == 2      # 8 heads on 3
+    one = mka.make_shape(1, 32, 1, 128)
+    assert mka.lib.mka_decode_paged(ctypes.byref(one), 1, None, pl, None, None, None, None, 0, None) == 2      # 32 heads per group
+    pl[1] = b.mka_paged_level(16, 16, 16, None, 64, 4, 0, 12, 2048, 256, 128, 8)                                # 12 rows per page
+    assert mka.lib.mka_decode_paged(ctypes.byref(dec), 2, None, pl, None, None, None, None, 0, None) == 2
+    pl[1] = b.mka_paged_level(16, 16, 16, None, 6400, 4, 0, 16, 2048, 256, 128, 8)                              # table too narrow
+    assert mka.lib.mka_decode_paged(ctypes.byref(dec), 2, None, pl, None, None, None, None, 0, None) == 2
+    pl[1] = b.mka_paged_level(16, 16, 16, None, 64, 4, 0, 16, 2048, 256, 128, 8)
+    assert mka.lib.mka_decode_paged(ctypes.byref(dec), 2, None, pl, None, None, None, None, 0, None) == 1      # null q
+    fwd = mka.make_shape(1, 8, 64, 128, window=8)
+    pl[1] = b.mka_paged_level(16, 16, 16, None, 64, 16, 0, 4, 2048, 256, 128, 8)                                # 4-row pages
+    assert mka.lib.mka_fwd_paged(ctypes.byref(fwd), 2, None, pl, None, None, None, None, 0, None) == 2
+    simt = mka.make_shape(1, 8, 64, 128, window=8, flags=1)
+    assert mka.lib.mka_fwd_paged(ctypes.byref(simt), 2, None, pl, None, None, None, None, 0, None) == 5
+    bad_group = mka.make_shape(1, 6, 4, 64, window=4, kv_heads=4)
+    lv = (b.mka_level * 3)()
+    assert mka.lib.mka_fwd(ctypes.byref(bad_group), None, lv, None, None, None, None, 0, None) == 2             # 6 heads on 4
+    # summary
+    assert mka.lib.mka_l2_summary(None, 1, 8, 20, 0, 0, 0.9, None, 0, None, None, 0, None) == 2                 # D % 8
+    assert mka.lib.mka_l2_summary(None, 1, 8, 64, 0, 1, 1.5, None, 0, None, None, 0, None) == 1                 # beta
+    assert mka.lib.mka_l2_summary(None, 0, 8, 64, 0, 0, 0.9, None, 0, None, None, 0, None) == 0                 # empty
+    # recall
+    assert mka.lib.mka_l3_index(None, 4, 2, 16, 96, 1, 1, 96, None, 64, None, None) == 2                        # d = 96
+    assert mka.lib.mka_l3_index(None, 4, 2, 16, 128, 1, 1, 128, None, 48, None, None) == 2                      # 48 bits
+    assert mka.lib.mka_l3_index(None, 0, 2, 16, 128, 1, 1, 128, None, 64, None, None) == 0                      # empty pool
+    assert mka.lib.mka_l3_retrieve(None, 1, 8, 3, 128, None, 64, None, None, None, 8, 8, 4, 16, None, None, None, None) == 2
+    assert mka.lib.mka_l3_retrieve(None, 1, 8, 2, 128, None, 64, None, None, None, 8, 8, 65, 16, None, None, None, None) == 2
+    assert mka.lib.mka_l3_retrieve(None, 1, 8, 2, 128, None, 64, None, None, None, 8, 8, 4, 16, None, None, None, None) == 1
+
+
+def test_summary_and_paged_workspace_queries(mka):
+    b = mka.binding
+    # 512 bytes + 8 bytes per (256-row segment, column)
+    assert mka.lib.mka_l2_summary_workspace_bytes(1, 32768, 4096, 0) == 512 + 128 * 4096 * 8
+    assert mka.lib.mka_l2_summary_workspace_bytes(2, 300, 64, 1) == 512 + 2 * 2 * 64 * 8
+    full = mka.lib.mka_l2_summary_workspace_bytes(1, 32768, 4096, 0)
+    assert mka.lib.mka_l2_summary_kernel_kind(1, 32768, 4096, 0, full) == 1
+    assert mka.lib.mka_l2_summary_kernel_kind(1, 32768, 4096, 0, full - 1) == 0          # not enough scratch
+    assert mka.lib.mka_l2_summary_kernel_kind(1, 400, 4096, 0, full) == 0                # short sequence
+    assert mka.lib.mka_l2_summary_kernel_kind(1, 32768, 4096, 1, 1 << 30) == 0           # fp32 with 128 strips: strip form
+    assert mka.lib.mka_l2_summary_kernel_kind(1, 32768, 1024, 1, 1 << 30) == 1           # fp32 with 32 strips
+    # the paged decode's split: chunks of a multiple of 128 rows, every partial slot accounted for
+    sh = mka.make_shape(4, 28, 1, 128)
+    n = (4096, 131072, 8192)
+    ws = mka.mka_decode_paged_workspace_bytes(sh, 4, n)
+    slots = (ws - 256) // (4 * 28 * 130 * 4)
+    assert (ws - 256) % (4 * 28 * 130 * 4) == 0 and 3 <= slots <= sum(-(-x // 128) for x in n)
+    # grouped heads in the dense decode take the same split as the paged decode
+    assert mka.mka_workspace_bytes(mka.make_shape(4, 28, 1, 128, kv_heads=4), n, b.MKA_WS_DECODE) == ws
