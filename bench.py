@@ -543,8 +543,8 @@ def oracle_sample(name, budget_rows=None):
         return {"value": bytes_ / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dt,
                 "sample": f"{len(heads)} of {cfg.B * cfg.H} (batch, head) pairs, all {cfg.T} rows each (numpy, one thread); router on all tokens"}
     # prefill / training: a few heads, a seeded sample of query rows
-    n_heads = 2 if budget_rows else 8          # the default sample is sized for roughly 10 s of host work
-    n_rows = budget_rows or 2048
+    n_heads = 2 if budget_rows else 8          # the default sample is sized for roughly 15 s of host work
+    n_rows = budget_rows or 4096
     n_rows = min(n_rows, cfg.T)
     heads = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(n_heads)]
     rows = np.sort(rng.choice(cfg.T, size=n_rows, replace=False))
