@@ -223,7 +223,7 @@ mka_status mka_decode_paged(const mka_shape* shape, int32_t H_kv, const void* q,
  * mka_l3_retrieve: per (sequence, KV head) the page table of the recalled chunks.
  *   q        [B, H, d] bf16;  codes from mka_l3_index with the same proj
  *   bank     int32 [B, bank_stride]: pool pages of each sequence's long-term chunks in time order; bank_len int32 [B]
- *            how many are in use (clamped to [0, max_bank]); max_bank (host) <= bank_stride, at most 32768
+ *            how many are in use (clamped to [0, max_bank]); max_bank (host) <= bank_stride, at most 98304 (the scores of a bank live in shared memory)
  *   R        chunks to recall, 1..64
  *   table    int32 [B, H_kv, R] out: recalled pool pages in bank order, unused slots 0
  *   n_sel    int32 [B] out or NULL: min(R, bank_len[b]);  rows int32 [B] out or NULL: n_sel * page_rows

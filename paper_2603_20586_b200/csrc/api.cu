@@ -431,7 +431,7 @@ mka_status mka_l3_retrieve(const void* q, int32_t B, int32_t H, int32_t H_kv, in
     if (d != 64 && d != 128) return MKA_ERR_SHAPE;
     if (bits != 32 && bits != 64 && bits != 128 && bits != 256) return MKA_ERR_SHAPE;
     if (R < 1 || R > 64 || page_rows <= 0) return MKA_ERR_SHAPE;
-    if (max_bank < 0 || max_bank > 32768 || bank_stride < max_bank) return MKA_ERR_SHAPE;
+    if (max_bank < 0 || max_bank > 98304 || bank_stride < max_bank) return MKA_ERR_SHAPE;
     if (B == 0 || H == 0) return MKA_OK;
     if (!q || !proj || !codes || !bank || !bank_len || !table) return MKA_ERR_ARG;
     cudaError_t e = launch_l3_retrieve(q, B, H, H_kv, d, proj, bits, codes, bank, bank_len, bank_stride, max_bank, R,

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from gpu_helpers import check, np64
-from mka_inputs import RECALL_CONFIGS, RecallConfig, make_recall
+from mka_inputs import RECALL_CONFIGS, RecallConfig, approx_normal, make_recall
 
 pytestmark = pytest.mark.gpu
 
@@ -94,3 +94,18 @@ def test_l3_rejects_bad_arguments(mka):
     with pytest.raises(mka.MkaError) as e:
         mka.mka_l3_retrieve(P["q"], 2, P["proj"], codes, P["bank"], P["bank_len"], 65, 8)  # R too large
     assert e.value.code == 2
+
+
+def test_recall_over_a_bank_of_70000_chunks(mka, orc):
+    """A bank longer than 65536 chunks (scores beyond 128 KB of shared memory); codes are planted by hand."""
+    B, H, H_kv, d, bits, R, n = 1, 2, 1, 64, 64, 8, 70000
+    g = torch.Generator().manual_seed(5)
+    codes = torch.randint(-2**31, 2**31 - 1, (n + 5, H_kv, bits // 32), generator=g, dtype=torch.int64).int().cuda()
+    proj = approx_normal(38, 1, 0, bits * d, 1.0, "cpu", torch.float32).view(bits, d).cuda()
+    q = approx_normal(38, 2, 0, B * H * d, 1.0, "cpu", torch.bfloat16).view(B, H, d).cuda()
+    bank = torch.randperm(n + 5, generator=g)[:n].int().view(1, n).cuda()
+    bank_len = torch.tensor([n], dtype=torch.int32, device="cuda")
+    table, n_sel, rows = mka.mka_l3_retrieve(q, H_kv, proj, codes, bank, bank_len, R, 16)
+    t_ref, n_ref = orc.l3_retrieve(q.float().cpu().numpy(), proj.cpu().numpy(), codes.cpu().numpy().view(np.uint32),
+                                   bank.cpu().numpy(), bank_len.cpu().numpy(), R, H_kv)
+    assert np.array_equal(table.cpu().numpy(), t_ref) and int(n_sel[0]) == R
