@@ -121,3 +121,51 @@ def test_paged_forward_with_identity_tables_is_the_dense_forward(orc):
     O, L = orc.fwd_paged(Q, pk, pv, tab, [n, n, n], pr, g, W, q_offset=2)
     Od, Ld = orc.fwd(Q, K, V, g, W, q_offset=2)
     assert np.array_equal(O, Od) and np.array_equal(L, Ld)
+
+
+def test_paged_forward_equals_eq5_written_out_through_the_tables(orc):
+    """Grouped heads, shuffled pools, a level with one page table per KV head, per-sequence row counts with one empty
+    sequence, a window shorter than the sequence and a query offset: every output row against Eq. 5 written out with
+    its own page walk and its own visibility rules."""
+    rng = np.random.default_rng(10)
+    B, H, H_kv, T, d, pr, W, q_off = 2, 6, 2, 7, 8, 4, 3, 2
+    rows = [np.array([9, 6]), np.array([8, 0]), np.array([9, 14])]       # level 2 of sequence 1 is empty
+    _, pk, pv, tab, _ = _case(rng, B, H, H_kv, d, pr, rows)
+    # long-term level: one table per KV head, the second head walks the same pages in reverse order
+    per_head = np.repeat(tab[2][:, None, :], H_kv, axis=1)
+    for b in range(B):
+        used = -(-int(rows[2][b]) // pr)
+        full = int(rows[2][b]) // pr                                       # only whole pages can swap places
+        per_head[b, 1, :full] = per_head[b, 1, :full][::-1].copy()
+        assert used > full >= 2
+    tables = [tab[0], tab[1], per_head]
+    Q = rng.normal(size=(B, H, T, d))
+    g = rng.random((B, T, 3)) + 0.05
+    g /= g.sum(-1, keepdims=True)
+    O, LSE = orc.fwd_paged(Q, pk, pv, tables, rows, pr, g, W, q_offset=q_off)
+    tau = 1.0 / np.sqrt(d)
+    for b in range(B):
+        for h in range(H):
+            kvh = h // 3                                  # heads 0-2 share KV head 0, heads 3-5 KV head 1
+            for t in range(T):
+                p = t + q_off
+                num, Z = np.zeros(d), 0.0
+                for l in range(3):
+                    for r in range(int(rows[l][b])):
+                        if l == 0 and not (p - W < r <= p):
+                            continue
+                        if l == 1 and not r <= p:
+                            continue
+                        page = tables[l][b, kvh, r // pr] if l == 2 else tables[l][b, r // pr]
+                        w = g[b, t, l] * np.exp(tau * Q[b, h, t] @ pk[l][page, kvh, r % pr])
+                        num += w * pv[l][page, kvh, r % pr]
+                        Z += w
+                assert Z > 0
+                assert np.allclose(O[b, h, t], num / Z, rtol=1e-12, atol=1e-12)
+                assert np.isclose(LSE[b, h, t], np.log(Z), rtol=1e-12)
+    # a table entry of KV head 1 that points somewhere else must change the heads of that KV head only
+    other = per_head.copy()
+    other[0, 1, 0] = per_head[1, 0, 0]                     # a full page of the other sequence: valid, different data
+    O2, _ = orc.fwd_paged(Q, pk, pv, [tab[0], tab[1], other], rows, pr, g, W, q_offset=q_off)
+    assert np.array_equal(O2[0, :3], O[0, :3]) and not np.array_equal(O2[0, 3:], O[0, 3:])
+    assert np.array_equal(O2[1], O[1])

@@ -205,6 +205,25 @@ def test_shift_invariance(orc):
     np.testing.assert_allclose(g1, g2, atol=1e-14)
 
 
+def test_score_shift_leaves_output_and_moves_lse(orc):
+    """A constant c added to EVERY score of a query row leaves O unchanged and moves LSE by c.  With one query row,
+    adding c q / (tau |q|^2) to every key of every level adds exactly c to each of its scores."""
+    rng = np.random.default_rng(30)
+    B, H, d, N, c = 1, 2, 6, (5, 7, 4), 2.75
+    Q = rng.standard_normal((B, H, 1, d))
+    K = [rng.standard_normal((B, H, n, d)) for n in N]
+    V = [rng.standard_normal((B, H, n, d)) for n in N]
+    gate = np.array([[[0.2, 0.5, 0.3]]])
+    tau = 1 / math.sqrt(d)
+    q = Q[:, :, 0]
+    delta = c * q / (tau * (q * q).sum(-1, keepdims=True))          # [B, H, d]
+    Ks = [k + delta[:, :, None, :] for k in K]
+    O1, L1 = orc.fwd(Q, K, V, gate, 1, decode=True)
+    O2, L2 = orc.fwd(Q, Ks, V, gate, 1, decode=True)
+    np.testing.assert_allclose(O2, O1, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(L2, L1 + c, rtol=1e-12, atol=1e-12)
+
+
 def test_nothing_visible_gives_zero_output(orc):
     rng = np.random.default_rng(31)
     B, H, T, d = 1, 1, 3, 4
