@@ -48,33 +48,47 @@ def load_peaks():
 
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures summarised under
-# profiles/.  The captures run the profiler-sized workloads (c3p, c4p, c5p: the same per-head geometry with fewer
-# heads / sequences); traffic grows in proportion to the number of (batch, head) pairs, so a full launch is the
-# captured figure times the ratio below.  None = not captured since the kernel last changed.
+# profiles/.  The captures run the profiler-sized workloads (c3p, c4p, c5p, ...: the same per-head geometry with fewer
+# heads / sequences); traffic grows in proportion to the number of units (batch x head pairs, sequences, KV heads), so
+# a full launch is the captured figure times the ratio below.  An entry is dropped (None) when its kernel changes
+# after the capture.
 NCU_TRAFFIC = {
-    # kernel: (bytes in the capture, (batch*head pairs of the capture))
-    "fwd_tc_kernel@c3": (376.360448e6 + 66.204160e6, 1 * 8),
-    "decode_partial_kernel@c4": (1.476463e9 + 5.216768e6, 2 * 32),
-    "bwd_dq_tc_kernel@c5": (220.282624e6 + 29.623808e6, 1 * 16),
-    "l2_summary_seg_kernel@s3": (100.972800e6 + 55.965184e6, 12288.0 / 32768.0),   # captured on 12288 of the 32768 tokens
-    "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8),
-    "decode_paged_kernel@g4": (293.713664e6 + 3.592192e6, 1 * 4),   # captured on one of the four sequences (g4p)
-    "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1),            # captured on one of the four sequences (r3p)
-    "bwd_dkv_tc_kernel@c5": (220.432640e6 + 115.097856e6, 1 * 16),
+    # kernel@workload: (bytes in the capture, units of the capture, summary file under profiles/)
+    "fwd_tc_kernel@c3": (376.360448e6 + 66.204160e6, 1 * 8, "fwd_tc_kernel_c3p.md"),
+    "decode_partial_kernel@c4": (1.476463e9 + 5.216768e6, 2 * 32, "decode_partial_kernel_c4p.md"),
+    "bwd_dq_tc_kernel@c5": (220.282624e6 + 29.623808e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
+    "l2_summary_seg_kernel@s3": (100.972800e6 + 55.965184e6, 12288.0 / 32768.0, "l2_summary_seg_kernel_s3p.md"),   # 12288 of the 32768 tokens
+    "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8, "fuse_kv_kernel_f3p.md"),
+    "decode_paged_kernel@g4": (293.713664e6 + 3.592192e6, 1 * 4, "decode_paged_kernel_g4p.md"),   # one of the four sequences (g4p)
+    "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1, "l3_index_kernel_r3p.md"),            # one of the four sequences (r3p)
+    "bwd_dkv_tc_kernel@c5": (220.432640e6 + 115.097856e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
 }
 
 
 def ncu_traffic(key, cfg):
+    """(bytes per full launch, where the figure comes from) or (None, None)."""
     ent = NCU_TRAFFIC.get(key)
     if ent is None:
-        return None
+        return None, None
     if key.startswith("l3_index"):
         units = cfg.B                                                      # one sequence's bank
     elif key.startswith("decode_paged"):
         units = cfg.B * cfg.H_kv                                           # one KV head of one sequence
     else:
         units = cfg.B if key.startswith("l2_summary") else cfg.B * cfg.H     # the summary's unit is a whole sequence
-    return ent[0] * units / ent[1]
+    ratio = units / ent[1]
+    return ent[0] * ratio, f"profiles/{ent[2]}, scaled x{ratio:.4g}"
+
+
+def sig(x, n=5):
+    """Rounds floats (recursively) to n significant digits: keeps the JSON line short."""
+    if isinstance(x, float):
+        return float(f"{x:.{n}g}") if x == x and abs(x) != float("inf") else x
+    if isinstance(x, dict):
+        return {k: sig(v, n) for k, v in x.items()}
+    if isinstance(x, (list, tuple)):
+        return [sig(v, n) for v in x]
+    return x
 
 
 def algorithmic_work(cfg):
@@ -190,6 +204,7 @@ class Leg:
                           "dV": [torch.empty_like(v) for v in self.V], "dG": torch.empty(B, T, 3, device=device),
                           "dW_r": torch.empty(D, 3, device=device), "db_r": torch.empty(3, device=device)}
             self.launches_per_step = 1 + 1 + (1 + 1 + 1 + 1) + 3   # router, fwd, bwd(prep,dq,dkv,dgate), router bwd
+            self.bwd_executed_ratio = 1.4           # the two-pass backward runs 14 d flops per pair for the method's 10 d
         else:
             self.launches_per_step = 2              # router, fwd
         self.ev = []
@@ -319,6 +334,13 @@ class Leg:
         r = [statistics.mean(a[i].elapsed_time(a[i + 1]) for a in self.ev) for i in range(3)]
         return {"router": r[0], "main": r[1], "bwd": r[2]}
 
+    def step_stats(self):
+        """Median and best device time of one whole step, and of its main kernel, over the recorded steps."""
+        whole = [a[0].elapsed_time(a[3]) for a in self.ev]
+        main = [a[1].elapsed_time(a[2]) for a in self.ev]
+        return {"n": len(whole), "step_median": statistics.median(whole), "step_best": min(whole),
+                "main_median": statistics.median(main), "main_best": min(main)}
+
 
 def timed_steps(leg, steps, warmup, dist=None):
     for _ in range(warmup):
@@ -344,70 +366,69 @@ def timed_steps(leg, steps, warmup, dist=None):
     return ms / steps
 
 
+def _hbm_roof(kernel, achieved, peaks, traffic):
+    t, src = traffic
+    roof = {"kernel": kernel, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"], "traffic": t,
+            "traffic_source": src}
+    if roof["frac"] > 1.0:
+        roof["note"] = "peak is a measured COPY rate (read + write); a read-mostly stream can exceed it"
+    return roof
+
+
+def _tensor_roof(kernel, achieved, peaks, traffic):
+    t, src = traffic
+    return {"kernel": kernel, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": achieved / peaks["bf16_tflops"], "frac_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+            "frac_datasheet": achieved / DATASHEET["bf16_tflops"], "traffic": t, "traffic_source": src}
+
+
 def leg_report(leg, ms_per_step, n_gpus, peaks):
     cfg, w, k = leg.cfg, leg.work, leg.kernel_ms()
+    none = (None, None)
+    tag = leg.name[:2]
     if leg.kind == "recall":
         # main = the index kernel; "bwd" holds the recall-list kernel plus the decode over the recalled chunks
-        achieved = w["index_bytes"] / (k["main"] * 1e-3) / 1e9
-        roof = {"kernel": "l3_index_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
-                "peak_source": peaks["source"], "traffic": ncu_traffic("l3_index_kernel@r3", cfg) if leg.name[:2] == "r3" else None}
-        value = n_gpus * w["index_bytes"] / (ms_per_step * 1e-3) / 1e9
-        unit, metric = "GB/s", "l3_recall_hbm_gbs"
+        work, unit, metric = w["index_bytes"], "GB/s", "l3_recall_hbm_gbs"
+        roof = _hbm_roof("l3_index_kernel", work / (k["main"] * 1e-3) / 1e9, peaks,
+                         ncu_traffic("l3_index_kernel@r3", cfg) if tag == "r3" else none)
     elif leg.kind == "paged":
-        achieved = w["decode_bytes"] / (k["main"] * 1e-3) / 1e9
-        roof = {"kernel": "decode_paged_kernel+decode_combine_kernel", "bound": "hbm", "achieved": achieved,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "frac_datasheet": achieved / DATASHEET["hbm_gbs"], "peak_source": peaks["source"],
-                "traffic": ncu_traffic("decode_paged_kernel@g4", cfg) if leg.name[:2] == "g4" else None}
-        value = n_gpus * w["decode_bytes"] / (ms_per_step * 1e-3) / 1e9
-        unit, metric = "GB/s", "decode_paged_hbm_gbs"
+        work, unit, metric = w["decode_bytes"], "GB/s", "decode_paged_hbm_gbs"
+        roof = _hbm_roof("decode_paged_kernel+decode_combine_kernel", work / (k["main"] * 1e-3) / 1e9, peaks,
+                         ncu_traffic("decode_paged_kernel@g4", cfg) if tag == "g4" else none)
     elif leg.kind == "summary":
-        achieved = w["summary_bytes"] / (k["main"] * 1e-3) / 1e9
-        roof = {"kernel": "l2_summary_seg_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
-                "peak_source": peaks["source"], "traffic": ncu_traffic("l2_summary_seg_kernel@s3", cfg) if leg.name[:2] == "s3" else None}
-        value = n_gpus * w["summary_bytes"] / (ms_per_step * 1e-3) / 1e9
-        unit, metric = "GB/s", "l2_summary_hbm_gbs"
+        work, unit, metric = w["summary_bytes"], "GB/s", "l2_summary_hbm_gbs"
+        roof = _hbm_roof("l2_summary_seg_kernel", work / (k["main"] * 1e-3) / 1e9, peaks,
+                         ncu_traffic("l2_summary_seg_kernel@s3", cfg) if tag == "s3" else none)
     elif leg.kind == "fuse":
-        achieved = w["fuse_bytes"] / (k["main"] * 1e-3) / 1e9
-        roof = {"kernel": "fuse_kv_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "frac_datasheet": achieved / DATASHEET["hbm_gbs"],
-                "peak_source": peaks["source"], "traffic": ncu_traffic("fuse_kv_kernel@f3", cfg) if leg.name[:2] == "f3" else None}
-        value = n_gpus * w["fuse_bytes"] / (ms_per_step * 1e-3) / 1e9
-        unit, metric = "GB/s", "route_fuse_hbm_gbs"
+        work, unit, metric = w["fuse_bytes"], "GB/s", "route_fuse_hbm_gbs"
+        roof = _hbm_roof("fuse_kv_kernel", work / (k["main"] * 1e-3) / 1e9, peaks,
+                         ncu_traffic("fuse_kv_kernel@f3", cfg) if tag == "f3" else none)
     elif leg.kind == "decode":
-        achieved = w["decode_bytes"] / (k["main"] * 1e-3) / 1e9
-        roof = {"kernel": "decode_partial_kernel+decode_combine_kernel", "bound": "hbm", "achieved": achieved,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "frac_datasheet": achieved / DATASHEET["hbm_gbs"], "peak_source": peaks["source"],
-                "traffic": ncu_traffic("decode_partial_kernel@c4", cfg) if leg.name[:2] == "c4" else None}
-        value = n_gpus * w["decode_bytes"] / (ms_per_step * 1e-3) / 1e9
-        unit, metric = "GB/s", "decode_hbm_gbs"
+        work, unit, metric = w["decode_bytes"], "GB/s", "decode_hbm_gbs"
+        roof = _hbm_roof("decode_partial_kernel+decode_combine_kernel", work / (k["main"] * 1e-3) / 1e9, peaks,
+                         ncu_traffic("decode_partial_kernel@c4", cfg) if tag == "c4" else none)
     else:
-        achieved = w["fwd_flops"] / (k["main"] * 1e-3) / 1e12
-        roof = {"kernel": "fwd_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                "frac_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
-                "frac_datasheet": achieved / DATASHEET["bf16_tflops"], "peak_source": peaks["source"],
-                "traffic": ncu_traffic("fwd_tc_kernel@c3", cfg) if leg.name[:2] == "c3" else None}
-        flops = w["fwd_flops"] + (w["bwd_flops"] if leg.kind == "train" else 0.0)
-        value = n_gpus * flops / (ms_per_step * 1e-3) / 1e12
+        work = w["fwd_flops"] + (w["bwd_flops"] if leg.kind == "train" else 0.0)
         unit, metric = "TFLOP/s", ("fwd_bwd_tflops" if leg.kind == "train" else "prefill_fwd_tflops")
+        roof = _tensor_roof("fwd_tc_kernel", w["fwd_flops"] / (k["main"] * 1e-3) / 1e12, peaks,
+                            ncu_traffic("fwd_tc_kernel@c3", cfg) if tag == "c3" else none)
+    scale = 1e9 if unit == "GB/s" else 1e12
+    value = n_gpus * work / (ms_per_step * 1e-3) / scale
+    st = leg.step_stats()
     rep = {"workload": leg.name, "metric": metric, "value": value, "unit": unit, "ms_per_step": ms_per_step,
-           "kernel_ms": k, "roofline": roof}
+           "steps": st["n"], "value_median": work / (st["step_median"] * 1e-3) / scale,
+           "value_best": work / (st["step_best"] * 1e-3) / scale, "kernel_ms": k, "roofline": roof}
     if leg.kind == "train":
         # the backward as a whole (prep, dQ kernel, dK/dV kernel, gate and router reductions) against the same peak;
         # "achieved" counts the 10*d flops per visible pair the method needs, not the 14*d the two-kernel form executes
         ach = w["bwd_flops"] / (k["bwd"] * 1e-3) / 1e12
         rep["bwd_tflops"] = ach
-        tq, tkv = ncu_traffic("bwd_dq_tc_kernel@c5", cfg), ncu_traffic("bwd_dkv_tc_kernel@c5", cfg)
-        rep["roofline_bwd"] = {"kernel": "bwd_dq_tc_kernel+bwd_dkv_tc_kernel", "bound": "tensor", "achieved": ach,
-                               "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                               "frac_sustained_peak": ach / peaks["bf16_tflops_sustained"],
-                               "frac_datasheet": ach / DATASHEET["bf16_tflops"], "executed_tflops": ach * 1.4,
-                               "peak_source": peaks["source"],
-                               "traffic": (tq + tkv) if (tq is not None and tkv is not None and leg.name[:2] == "c5") else None}
+        tq, sq = ncu_traffic("bwd_dq_tc_kernel@c5", cfg)
+        tkv, _ = ncu_traffic("bwd_dkv_tc_kernel@c5", cfg)
+        both = tq is not None and tkv is not None and tag == "c5"
+        rep["roofline_bwd"] = _tensor_roof("bwd_dq_tc_kernel+bwd_dkv_tc_kernel", ach, peaks, ((tq + tkv), sq) if both else none)
+        rep["roofline_bwd"]["executed_tflops"] = ach * leg.bwd_executed_ratio
     return rep
 
 
@@ -485,11 +506,11 @@ def oracle_sample_recall(name):
 
 
 def oracle_sample(name, budget_rows=None):
+    """Times the CPU oracle, as it stands, on a bounded seeded sample of workload `name`."""
     if name in PAGED_CONFIGS:
         return oracle_sample_paged(name)
     if name in RECALL_CONFIGS:
         return oracle_sample_recall(name)
-    """Times the CPU oracle, as it stands, on a bounded seeded sample of workload `name`."""
     from oracle import mka_oracle as orc
     orc.build()
     cfg = CONFIGS[name]
@@ -640,8 +661,10 @@ def main():
     clocks = sampler.stop()
     rep = leg_report(leg, ms, world, peaks)
     launches = leg.launches_per_step * args.steps
-    out = dict(base, value=rep["value"], unit=rep["unit"], ms_per_step=ms, roofline=rep["roofline"], kernel_ms=rep["kernel_ms"],
+    out = dict(base, value=rep["value"], unit=rep["unit"], ms_per_step=ms, value_median=rep["value_median"] * world,
+               value_best=rep["value_best"] * world, roofline=rep["roofline"], kernel_ms=rep["kernel_ms"],
                clocks=clocks, gpu_launches=launches, n_gpus=world)
+    out["roofline"]["peak_source"] = peaks["source"]
     if "bwd_tflops" in rep:
         out["bwd_tflops"] = rep["bwd_tflops"]
         out["roofline_bwd"] = rep["roofline_bwd"]
@@ -661,20 +684,24 @@ def main():
         out["e2e"] = {"value": ev, "unit": rep["unit"], "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
     del leg
     torch.cuda.empty_cache()
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = oracle_sample(args.workload)
+    # The other configurations, each for --steps timed steps.  The two the headline metric names besides prefill --
+    # training (c5) and decode (c4) -- come last, so that they end the line.
     legs = []
     if world == 1:
-        for name in [x for x in args.legs.split(",") if x and x != args.workload]:
+        wanted = [x for x in args.legs.split(",") if x and x != args.workload]
+        order = {n: i for i, n in enumerate(["r3", "g4", "s3", "f3", "c2", "c5", "c4"])}
+        wanted.sort(key=lambda n: order.get(n[:2], -1))
+        for name in wanted:
             l2 = Leg(name, dev)
-            k = max(3, min(args.steps, 5)) if name != "c4" else max(3, min(args.steps, 20))
-            ms2 = timed_steps(l2, k, 3)
+            ms2 = timed_steps(l2, max(3, args.steps), max(3, args.warmup))
             legs.append(leg_report(l2, ms2, 1, peaks))
             del l2
             torch.cuda.empty_cache()
     out["legs"] = legs
     if rank == 0:
-        if not args.no_cpu_baseline and world == 1:
-            out["cpu_baseline"] = oracle_sample(args.workload)
-        print(json.dumps(out))
+        print(json.dumps(sig(out)))
     if dist is not None:
         dist.destroy_process_group()
 

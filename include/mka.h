@@ -63,6 +63,11 @@ typedef enum { MKA_ROUTE_SOFT = 0, MKA_ROUTE_UNIFORM = 1, MKA_ROUTE_TOP1 = 2, MK
 
 /* mka_shape.flags */
 #define MKA_FLAG_FORCE_SIMT 1u   /* run the CUDA-core kernels even where a tensor-core kernel exists */
+#define MKA_FLAG_TEST_STALL 0x80000000u /* test hook of mka_fwd (tensor-core kernel, dense levels): the loader of every
+                                           CTA leaves out its last key tile, so the wait for that tile runs into the
+                                           limit of mka_set_wait_limit_us and the call ends with MKA_ERR_TIMEOUT in
+                                           the status word; O and LSE of such a call are invalid.  Exists so that
+                                           the give-up path can be exercised without a fault or a hang. */
 
 /* which = argument of mka_workspace_bytes */
 #define MKA_WS_FWD 0
@@ -191,20 +196,22 @@ typedef struct mka_paged_level {
  *       chunks of a multiple of 128 rows (at most 8192), chosen so that the grid makes few rounds of the resident CTAs
  * d must be 64 or 128; pools 16-byte aligned with strides that are multiples of 8 elements.
  */
+size_t mka_decode_paged_workspace_bytes(const mka_shape* shape, int32_t H_kv, const int64_t n_level[3]);
+mka_status mka_decode_paged(const mka_shape* shape, int32_t H_kv, const void* q, const mka_paged_level L[3],
+                            const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
+
 /*
  * Fused forward of mka_fwd over paged levels (prefill, or a chunk of it, against a paged KV cache) with grouped-query
  * sharing: same result as mka_fwd on the gathered levels with shape->kv_heads = H_kv.  Sequence b has rows[b] rows on
  * level l (L[l].n for all when rows is NULL); all sequences share T and q_offset.  page_rows must be a power of two
- * >= 8; pool_pages must be set; rows of a sequence's last page past its length must hold finite values (they are
- * loaded and masked, not skipped).
+ * >= 8; pool_pages must be set.  Rows of a sequence's last page after its last row may hold anything (NaN and Inf
+ * included): the page is copied whole, the key rows are masked and the value rows are cleared in shared memory before
+ * the product reads them.  Pages with no valid row are never read.
  * bf16, MKA_MODE_FAST, d in {64, 128} only (the TMA + tcgen05 kernel; a 128-row key tile is assembled from one box
  * per page); anything else returns MKA_ERR_UNSUPPORTED.  ws: at least 256 bytes (status word).
  */
 mka_status mka_fwd_paged(const mka_shape* shape, int32_t H_kv, const void* Q, const mka_paged_level L[3],
                          const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
-size_t mka_decode_paged_workspace_bytes(const mka_shape* shape, int32_t H_kv, const int64_t n_level[3]);
-mka_status mka_decode_paged(const mka_shape* shape, int32_t H_kv, const void* q, const mka_paged_level L[3],
-                            const float* gate, void* O, float* LSE, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * L3 recall (Alg. 2 step 4 "L3 <- Retrieve(Q_h)"; the method section's vectorized hashing with chunk-based recall; the
@@ -246,6 +253,10 @@ mka_status mka_l3_retrieve(const void* q, int32_t B, int32_t H, int32_t H_kv, in
  *   O, LSE: outputs of mka_fwd;  dO [B,H,T,d];  R [B*T, D] router input in r_dtype (NULL skips dW_r, db_r)
  *   dQ [B,H,T,d];  dL[3] gradient destinations (a level with n == 0 is skipped);  dG [B,T,3] f32;
  *   dW_r [D,3] f32 or NULL;  db_r [3] f32 or NULL.
+ * dG is the logit gradient of a gate that is a softmax of the logits (MKA_ROUTE_SOFT; for TOP1 / TOP2 the renormalised
+ * softmax over the kept levels, whose dropped levels get dG = 0 because their gate is 0).  dW_r = R^T dG and
+ * db_r = sum dG follow from that; with MKA_ROUTE_UNIFORM the gate does not depend on W_r, so the true dW_r, db_r are 0
+ * and a caller training that variant passes dW_r = db_r = NULL.
  * bf16 with d in {64,128} runs the TMA + tcgen05 kernels (one pass that owns query tiles for dQ and dG, one
  * pass that owns key tiles for dK and dV; scores are recomputed in each, nothing is accumulated atomically);
  * f32, other head widths and MKA_FLAG_FORCE_SIMT run the CUDA-core kernels.  Both are deterministic.
@@ -287,6 +298,10 @@ mka_status mka_fuse_kv_paged(int32_t B, int32_t H, int64_t n, int32_t d, int32_t
 
 /* Causal summaries of mka_l2_summary. */
 typedef enum { MKA_SUMMARY_MEAN = 0, MKA_SUMMARY_EMA = 1 } mka_summary;
+/* Test hook, OR-ed into `kind` (segmented form only): segment 1 of every column strip never publishes its carried
+ * state, so the look-back of the later segments runs into the limit of mka_set_wait_limit_us and the call ends with
+ * MKA_ERR_TIMEOUT in the status word; M2 and state of such a call are invalid. */
+#define MKA_SUMMARY_TEST_STALL 0x40000000
 
 /*
  * L2 session summary (Alg. 1, the loop "M_2[t] <- Summary(X[:, 1:t, :])", named there as "prefix mean or EMA";
@@ -329,9 +344,13 @@ int32_t mka_l2_summary_kernel_kind(int32_t B, int64_t T, int32_t D, int32_t dtyp
  *   - Limit: B * H * total_chunks * (d + 2) floats (total_chunks from mka_decode_plan) must fit in
  *     mka_decode_static_max_bytes() = 8 MiB; larger problems are rejected with MKA_ERR_WORKSPACE and
  *     nothing is launched.  (For d = 128 that is 16131 chunk partials, e.g. 32 heads x 516k cached rows.)
- *   - The array costs 8 MiB on every GPU that loads the library, for the life of the process.
+ *   - The array costs 8 MiB on every GPU that runs a decode kernel of this library, for the life of the
+ *     process.  The CUDA runtime sets it aside when this part of the library is first used on a device (the
+ *     first decode call, or the address look-up below), not when the library is loaded; on a device whose
+ *     memory is already exhausted that first use fails and the call returns MKA_ERR_CUDA.
  *   - The first call on each device looks up the array's device address (with that device current)
- *     and remembers it; make that first call during set-up, before any stream capture begins.
+ *     and remembers it; make that first call during set-up, before any stream capture begins.  The
+ *     remembered address does not survive a cudaDeviceReset of that device.
  *   - All calls on one device share the one array and it keeps whatever the last call wrote.  Nothing
  *     in it needs clearing between calls (every slot that is read was written by the same call), but
  *     two calls whose kernels overlap on the GPU -- different streams, no ordering between them --
@@ -359,6 +378,13 @@ int32_t mka_bwd_kernel_kind(const mka_shape* shape, const mka_level L[3], const 
  * `ws` left there: MKA_OK, or MKA_ERR_TIMEOUT when a bounded wait inside a kernel gave up (the
  * kernel then released its resources and returned; outputs of that call are invalid). */
 mka_status mka_device_status(const void* ws, void* stream);
+
+/* Limit, in microseconds, of every wait inside the kernels (a warp waiting for a tile to land, for another warp's
+ * result, for an earlier segment's state).  A wait that reaches it gives up: the CTA releases what it holds, the kernel
+ * returns and the status word of the call's workspace reads MKA_ERR_TIMEOUT.  Default 1 000 000 (one second, far above
+ * anything a healthy launch needs); 0 restores the default; values are clamped to [100, 10 000 000].  Process-wide,
+ * read when a call is made.  Returns the previous value.  Host function, no CUDA call. */
+uint32_t mka_set_wait_limit_us(uint32_t us);
 
 #ifdef __cplusplus
 }

@@ -19,14 +19,16 @@ MKA_BF16, MKA_F32 = 0, 1
 MKA_MODE_FAST, MKA_MODE_FULL = 0, 1
 MKA_ROUTE_SOFT, MKA_ROUTE_UNIFORM, MKA_ROUTE_TOP1, MKA_ROUTE_TOP2 = 0, 1, 2, 3
 MKA_FLAG_FORCE_SIMT = 1
+MKA_FLAG_TEST_STALL = 0x80000000
 MKA_SUMMARY_MEAN, MKA_SUMMARY_EMA = 0, 1
+MKA_SUMMARY_TEST_STALL = 0x40000000
 MKA_WS_FWD, MKA_WS_DECODE, MKA_WS_BWD = 0, 1, 2
 TILE = 128
 
 EXPORTS = ["mka_status_str", "mka_router", "mka_workspace_bytes", "mka_fwd", "mka_decode", "mka_bwd",
            "mka_decode_plan", "mka_fwd_tile_range", "mka_device_status", "mka_fwd_kernel_kind",
            "mka_bwd_kernel_kind", "mka_fuse_kv", "mka_l2_summary", "mka_l2_summary_workspace_bytes", "mka_l2_summary_kernel_kind", "mka_decode_static", "mka_decode_static_max_bytes",
-           "mka_decode_paged", "mka_decode_paged_workspace_bytes", "mka_l3_index", "mka_l3_retrieve", "mka_fwd_paged", "mka_fuse_kv_paged"]
+           "mka_decode_paged", "mka_decode_paged_workspace_bytes", "mka_l3_index", "mka_l3_retrieve", "mka_fwd_paged", "mka_fuse_kv_paged", "mka_set_wait_limit_us"]
 
 
 class MkaError(RuntimeError):
@@ -106,10 +108,12 @@ def _load() -> ctypes.CDLL:
     lib.mka_l2_summary_kernel_kind.argtypes = [i32, i64, i32, i32, ctypes.c_size_t]
     lib.mka_l2_summary.argtypes = [vp, i32, i64, i32, i32, i32, ctypes.c_float, vp, i64, vp, vp, ctypes.c_size_t, vp]
     lib.mka_bwd_kernel_kind.argtypes = [ctypes.POINTER(mka_shape), ctypes.POINTER(mka_level), vp]
+    lib.mka_set_wait_limit_us.argtypes = [ctypes.c_uint32]
     for name in EXPORTS:
         if name not in ("mka_status_str", "mka_workspace_bytes", "mka_decode_static_max_bytes", "mka_l2_summary_workspace_bytes",
-                        "mka_decode_paged_workspace_bytes"):
+                        "mka_decode_paged_workspace_bytes", "mka_set_wait_limit_us"):
             getattr(lib, name).restype = ctypes.c_int
+    lib.mka_set_wait_limit_us.restype = ctypes.c_uint32
     return lib
 
 
@@ -438,3 +442,8 @@ def mka_bwd_kernel_kind(shape: mka_shape, K, V) -> int:
 
 def mka_device_status(ws: torch.Tensor, stream=None) -> int:
     return int(lib.mka_device_status(_ptr(ws), _stream(stream)))
+
+
+def mka_set_wait_limit_us(us: int) -> int:
+    """Sets the limit of the kernels' internal waits (microseconds; 0 = the default of one second); returns the old one."""
+    return int(lib.mka_set_wait_limit_us(int(us)))

@@ -2,9 +2,23 @@
 // table, forward tile ranges), workspace layout, and dispatch to the kernels.  See include/mka.h.
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 using namespace mka;
+
+// Process-wide limit of the device-side waits, in microseconds.
+static std::atomic<uint32_t> g_wait_limit_us{1000000u};
+unsigned long long mka::wait_limit_ns() { return 1000ull * g_wait_limit_us.load(std::memory_order_relaxed); }
+
+extern "C" uint32_t mka_set_wait_limit_us(uint32_t us) {
+    if (us == 0) us = 1000000u;
+    if (us < 100u) us = 100u;
+    if (us > 10000000u) us = 10000000u;
+    return g_wait_limit_us.exchange(us, std::memory_order_relaxed);
+}
 
 namespace {
 
@@ -183,6 +197,7 @@ mka_status mka_fwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
     p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s);
     p.mode = s->mode; p.decode = 0; p.kv_group = kv_group_of(s);
+    p.test_stall = (s->flags & MKA_FLAG_TEST_STALL) ? 1 : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;
     cudaError_t e;
@@ -592,6 +607,8 @@ mka_status mka_fuse_kv_paged(int32_t B, int32_t H, int64_t n, int32_t d, int32_t
 mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_t dtype, int32_t kind, float beta, float* state,
                           int64_t n_prev, void* M2, void* ws, size_t ws_bytes, void* stream) {
     if (dtype != MKA_BF16 && dtype != MKA_F32) return MKA_ERR_ARG;
+    const int32_t stall = kind & MKA_SUMMARY_TEST_STALL;
+    kind &= ~MKA_SUMMARY_TEST_STALL;
     if (kind != MKA_SUMMARY_MEAN && kind != MKA_SUMMARY_EMA) return MKA_ERR_ARG;
     if (B < 0 || T < 0 || D < 0 || n_prev < 0 || B > 65535) return MKA_ERR_SHAPE;
     if (T > 0x7fffff00LL) return MKA_ERR_SHAPE;
@@ -608,7 +625,7 @@ mka_status mka_l2_summary(const void* X, int32_t B, int64_t T, int32_t D, int32_
     // busy however few column strips there are; otherwise one CTA walks each strip from end to end.
     const bool segmented = ws && (reinterpret_cast<uintptr_t>(ws) & 15) == 0 && mka_l2_summary_kernel_kind(B, T, D, dtype, ws_bytes) == 1;
     cudaError_t e = segmented
-        ? launch_l2_summary_seg(X, M2, state, n_prev > 0 ? 1 : 0, n_prev, B, T, D, dtype, kind, beta,
+        ? launch_l2_summary_seg(X, M2, state, n_prev > 0 ? 1 : 0, n_prev, B, T, D, dtype, kind | stall, beta,
                                 static_cast<unsigned int*>(ws), static_cast<char*>(ws) + kWsHeader, cs)
         : launch_l2_summary(X, M2, state, n_prev > 0 ? 1 : 0, n_prev, B, T, D, dtype, kind, beta,
                             static_cast<unsigned int*>(ws), cs);

@@ -56,6 +56,7 @@ struct BwdTcParams {
     float scale, scale_log2;
     int kv_tiles[3];          // 128-row key tiles per level
     unsigned int* status;
+    unsigned long long wait_limit_ns;
 };
 
 template <int DH>
@@ -192,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
     float (*gsm)[6] = reinterpret_cast<float (*)[6]>(sQ); // epilogue scratch; Q is dead once the last S product has completed
     __shared__ BwdBarriers bar;
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    __shared__ WaitCtl wait_ctl;
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
@@ -203,7 +204,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
     const long long m_last = (m0 + kBlk - 1 < p.T - 1) ? m0 + kBlk - 1 : p.T - 1;
 
     if (tid == 0) {
-        abort_flag = 0;
+        wait_ctl.abort = 0;
+        wait_ctl.limit_ns = p.wait_limit_ns;
         mbar_init(&bar.fixed_full, 1);
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1);
@@ -222,7 +224,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
-    volatile int* abortp = &abort_flag;
+    volatile WaitCtl* abortp = &wait_ctl;
 
     int first[3], end[3];
 #pragma unroll
@@ -439,7 +441,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
 
     tc_fence_before();
     __syncthreads();
-    if (tid == 0 && abort_flag) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
+    if (tid == 0 && wait_ctl.abort) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
 }
 
@@ -457,7 +459,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     float* sStat = reinterpret_cast<float*>(sdO + C::kStages * C::kTile);     // kStages x {D[128], bias[128]}
     __shared__ BwdBarriers bar;
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    __shared__ WaitCtl wait_ctl;
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
@@ -484,7 +486,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     const int E = Eq * p.kv_group;                          // the stream: head by head, each head's tiles in order
 
     if (tid == 0) {
-        abort_flag = 0;
+        wait_ctl.abort = 0;
+        wait_ctl.limit_ns = p.wait_limit_ns;
         mbar_init(&bar.fixed_full, 1);
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1); }
         mbar_init(&bar.s_full[0], 1);
@@ -500,7 +503,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
-    volatile int* abortp = &abort_flag;
+    volatile WaitCtl* abortp = &wait_ctl;
 
     if (warp == kProducerWarp) {
         if (lane == 0 && E > 0) {
@@ -700,7 +703,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
 
     tc_fence_before();
     __syncthreads();
-    if (tid == 0 && abort_flag) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
+    if (tid == 0 && wait_ctl.abort) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
 }
 
@@ -736,6 +739,7 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
     p.window = bp.window; p.q_offset = bp.q_offset;
     p.scale = bp.scale; p.scale_log2 = bp.scale * kLog2e;
     p.status = status_word;
+    p.wait_limit_ns = wait_limit_ns();
 
     // both kernels move 128-row tiles (box = 64 columns x 128 rows)
     {

@@ -44,6 +44,7 @@ struct FwdParams {
     int mode;
     int decode;         // every row visible
     int kv_group;       // query heads per KV head (>= 1): head h reads KV head h / kv_group
+    int test_stall;     // MKA_FLAG_TEST_STALL (tensor-core forward, dense levels)
     const PagedLevelDev* paged;   // host array of 3, or null: the levels are page pools (tensor-core forward only; L[l].n still holds the rows)
 };
 

@@ -274,7 +274,10 @@ float* g_static_scratch_ptr[kMaxDevices];       // device address of the array, 
 std::mutex g_static_scratch_mutex;
 
 // In host code the array's name is only a handle; the address a kernel can use has to be asked for,
-// once per device and with that device current.
+// once per device and with that device current.  With CUDA's lazy module loading that request (or the first
+// launch from this file) is also the moment the 8 MiB are really taken on that device, so it can fail when the
+// device has no memory left: the caller then sees MKA_ERR_CUDA from its first call.  The remembered address
+// belongs to the device's current context and is not refreshed after a cudaDeviceReset.
 cudaError_t static_scratch_address(float** out) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -306,6 +309,7 @@ extern "C" mka_status mka_decode_static(const mka_shape* s, const void* q, const
     if (s->dtype != MKA_BF16 || s->mode != MKA_MODE_FAST) return MKA_ERR_UNSUPPORTED;
     if (s->B < 0 || s->H < 0 || s->T != 1) return MKA_ERR_SHAPE;
     if (s->d != 64 && s->d != 128) return MKA_ERR_SHAPE;
+    if (s->kv_heads < 0 || (s->kv_heads > 0 && (s->H % s->kv_heads != 0))) return MKA_ERR_SHAPE;
     int64_t n_level[3];
     for (int l = 0; l < 3; ++l) {
         n_level[l] = L[l].n;
@@ -336,7 +340,6 @@ extern "C" mka_status mka_decode_static(const mka_shape* s, const void* q, const
         p.n_chunks[l] = plan.n_chunks[l];
     }
     p.B = s->B; p.H = s->H; p.d = s->d;
-    if (s->kv_heads < 0 || (s->kv_heads > 0 && (s->H % s->kv_heads != 0))) return MKA_ERR_SHAPE;
     p.kv_group = s->kv_heads > 0 ? s->H / s->kv_heads : 1;
     p.scale = s->scale > 0.f ? s->scale : 1.0f / sqrtf((float)s->d);
     p.chunk_rows = plan.chunk_rows;

@@ -50,6 +50,8 @@ struct TcParams {
     int window, q_offset;
     float scale_log2;
     unsigned int* status;
+    unsigned long long wait_limit_ns;
+    int test_stall;          // test hook (MKA_FLAG_TEST_STALL): the producer leaves out the last key tile of every CTA
     // paged levels: a 128-row key tile is assembled from boxes of box_rows rows, one page-table look-up per box
     int paged;
     const int* table[3];
@@ -101,7 +103,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     uint8_t* sV = sK + C::kStages * C::kTileBytes;        // kStages tiles
     __shared__ Barriers bar;
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    __shared__ WaitCtl wait_ctl;
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
@@ -111,7 +113,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     const long long m_last = (m0 + kNumQ * kTileM - 1 < p.T - 1) ? m0 + kNumQ * kTileM - 1 : p.T - 1;
 
     if (tid == 0) {
-        abort_flag = 0;
+        wait_ctl.abort = 0;
+        wait_ctl.limit_ns = p.wait_limit_ns;
         mbar_init(&bar.q_full, 1);
         for (int s = 0; s < 4; ++s) {
             mbar_init(&bar.k_full[s], 1); mbar_init(&bar.k_empty[s], 1);
@@ -131,7 +134,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
-    volatile int* abortp = &abort_flag;
+    volatile WaitCtl* abortp = &wait_ctl;
 
     // rows of the three levels for this sequence
     long long nl[3];
@@ -227,6 +230,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             const int kvh = h / p.kv_group;
             for (int l = 0; l < 3 && ok; ++l) {
                 for (int kt = first[l]; kt < end[l]; ++kt) {
+                    if (p.test_stall && issued_k == E - 1) break;      // test hook: the last tile never arrives
                     const int e = issued_k;
                     const int s = e % C::kStages;
                     const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
@@ -267,6 +271,40 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                            C::kIdescQK, k > 0);
                 mma_commit_elect(&bar.s_full[q]);
             };
+            // Paged levels: the page that holds a level's last row is copied whole, so the rows after that row arrive
+            // with whatever the pool holds there (a recycled page, never-written memory).  Their weights are exactly 0,
+            // but 0 x NaN or 0 x Inf would still poison the accumulator: those V rows are cleared here, after the
+            // copy has landed and before the product reads them.  (K needs nothing: masked scores are overwritten.)
+            int scrub_e[3] = {-1, -1, -1}, scrub_r0[3] = {0, 0, 0}, scrub_r1[3] = {0, 0, 0};
+            if (kPaged) {
+                int e0 = 0;
+#pragma unroll
+                for (int l = 0; l < 3; ++l) {
+                    const int tiles = end[l] - first[l];
+                    const int tail = (int)(nl[l] % kTileN);
+                    if (tiles > 0 && tail != 0 && (long long)end[l] * kTileN > nl[l]) {
+                        const int rpb = p.box_rows[l];
+                        scrub_e[l] = e0 + tiles - 1;
+                        scrub_r0[l] = tail;
+                        scrub_r1[l] = (tail + rpb - 1) / rpb * rpb;      // end of the box that straddles the level's end
+                    }
+                    e0 += tiles;
+                }
+            }
+            auto scrub_v = [&](int e, int s) {
+                if (!kPaged) return;
+#pragma unroll
+                for (int l = 0; l < 3; ++l) {
+                    if (e != scrub_e[l]) continue;
+                    const int vecs = (scrub_r1[l] - scrub_r0[l]) * 8;      // 16-byte vectors per 64-column panel
+                    for (int pn = 0; pn < C::kPanels; ++pn) {
+                        uint4* base = reinterpret_cast<uint4*>(sV + s * C::kTileBytes + pn * kPanelBytes + scrub_r0[l] * 128);
+                        for (int i = lane; i < vecs; i += 32) base[i] = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
+            };
             auto issue_pv = [&](int q, int s, bool accumulate) {
                 const uint32_t va = v_lo + s * (C::kTileBytes >> 4);
 #pragma unroll
@@ -298,6 +336,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                         mma_commit_elect(&bar.k_empty[sn]);
                     }
                     if (!mbar_wait_warp(&bar.v_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) { ok = false; break; }
+                    scrub_v(e, s);
 #pragma unroll
                     for (int q = 0; q < kNumQ; ++q) {
                         if (!mbar_wait_warp(&bar.p_full[q], (uint32_t)e & 1u, abortp)) { ok = false; break; }
@@ -324,6 +363,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 issue_qk(1, s);
                 mma_commit_elect(&bar.k_empty[s]);
                 if (!mbar_wait_warp(&bar.v_full[s], ph, abortp)) { ok = false; break; }
+                scrub_v(e, s);
                 if (!mbar_wait_warp(&bar.p_full[0], (uint32_t)e & 1u, abortp)) { ok = false; break; }
                 tc_fence_after();
                 issue_pv(0, s, e > 0);
@@ -483,7 +523,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
 
     tc_fence_before();
     __syncthreads();
-    if (tid == 0 && abort_flag) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
+    if (tid == 0 && wait_ctl.abort) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
 }
 
@@ -525,6 +565,8 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
     p.window = fp.window; p.q_offset = fp.q_offset;
     p.scale_log2 = fp.scale * kLog2e;
     p.status = status_word;
+    p.wait_limit_ns = wait_limit_ns();
+    p.test_stall = fp.test_stall;
     auto kern = fp.paged ? fwd_tc_kernel<DH, true> : fwd_tc_kernel<DH, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<DH>::kSmemBytes);
     if (e != cudaSuccess) return e;

@@ -28,6 +28,7 @@ struct SummaryParams {
     int use_state;         // state holds a carried value on entry
     int stages;            // depth of the tile ring
     unsigned int* status;  // may be null
+    unsigned long long wait_limit_ns;
 };
 
 // two adjacent columns of a row at once
@@ -66,7 +67,7 @@ __global__ void __launch_bounds__(kSumThreads, 3) l2_summary_kernel(const __grid
     __shared__ float2 part[G][kNP];
     __shared__ float2 carry[kNP];
     __shared__ uint64_t full[kSumMaxStages];
-    __shared__ int abort_flag;
+    __shared__ WaitCtl wait_ctl;
 
     const int tid = threadIdx.x;
     const int c = tid % kNP, g = tid / kNP;           // column pair, row group
@@ -77,7 +78,8 @@ __global__ void __launch_bounds__(kSumThreads, 3) l2_summary_kernel(const __grid
     const float beta = p.beta, omb = 1.f - p.beta;
 
     if (tid == 0) {
-        abort_flag = 0;
+        wait_ctl.abort = 0;
+        wait_ctl.limit_ns = p.wait_limit_ns;
         for (int s = 0; s < kSumMaxStages; ++s) mbar_init(&full[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -91,7 +93,7 @@ __global__ void __launch_bounds__(kSumThreads, 3) l2_summary_kernel(const __grid
         carry[tid] = v;
     }
     __syncthreads();
-    volatile int* abortp = &abort_flag;
+    volatile WaitCtl* abortp = &wait_ctl;
     // a box of the tensor map holds at most 256 rows: taller tiles arrive as consecutive boxes on the same barrier
     constexpr int kBoxRows = kRows > 256 ? 256 : kRows;
     auto load_tile = [&](uint8_t* dst, int row0, uint64_t* bar) {
@@ -231,7 +233,7 @@ cudaError_t launch_l2_summary(const void* X, void* M2, float* state, int use_sta
     if (!tensor_map_encoder_available()) return cudaErrorNotSupported;
     SummaryParams p;
     p.M2 = M2; p.state = state; p.T = T; p.n_prev = n_prev; p.B = B; p.D = D; p.kind = kind; p.beta = beta;
-    p.use_state = use_state; p.status = status;
+    p.use_state = use_state; p.status = status; p.wait_limit_ns = wait_limit_ns();
     // Strips as wide as possible (whole 128-byte lines per row are kindest to DRAM) while most SMs still get a CTA;
     // the fewer CTAs share an SM, the deeper each one's ring of tiles in flight.
     const long long want = 120;

@@ -35,6 +35,8 @@ struct SegParams {
     float beta;
     int use_state;
     unsigned int* status;
+    unsigned long long wait_limit_ns;
+    int test_stall;          // test hook (MKA_SUMMARY_TEST_STALL): segment 1 of every strip never publishes its records
 };
 
 template <typename T> struct Pair2;
@@ -107,7 +109,7 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
     __shared__ float carry[kNC];
     __shared__ float a_pow[RG + 1];                            // beta^j, j = 0..RG (EMA)
     __shared__ uint64_t full;
-    __shared__ int abort_flag;
+    __shared__ WaitCtl wait_ctl;
     __shared__ unsigned place_s;
     __shared__ int pending_s;                                  // parity of the newest load's barrier phase, or -1 before any load
 
@@ -116,7 +118,7 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
     const int Tn = (int)p.T;
     const float beta = p.beta, omb = 1.f - p.beta;
     const unsigned total = (unsigned)p.S * p.B * p.strips;
-    volatile int* abortp = &abort_flag;
+    volatile WaitCtl* abortp = &wait_ctl;
     float a_rg = 1.f;                                          // beta^RG, beta^kSegRows
     if (kEma) {
 #pragma unroll
@@ -134,7 +136,8 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
         a_pow[tid] = a;
     }
     if (tid == 0) {
-        abort_flag = 0;
+        wait_ctl.abort = 0;
+        wait_ctl.limit_ns = p.wait_limit_ns;
         pending_s = -1;
         mbar_init(&full, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,7 +226,7 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
                     }
                 }
             } else {
-                if (col_ok) st_rec2(my_rec + 2 * lane, kFlagAggregate, tot);
+                if (col_ok && !(p.test_stall && seg == 1)) st_rec2(my_rec + 2 * lane, kFlagAggregate, tot);
                 // Look back eight segments at a time (the segment at distance d = d0 + k is record k of the window)
                 // until every column has met an INCLUSIVE record with nothing unpublished nearer than it.
                 // Folding runs from the far end, state(d) = a * state(d + 1) + b(d), restarting at any inclusive
@@ -251,7 +254,7 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
                     }
                     const int kk = incl_all ? __ffs(incl_all) - 1 : 7;
                     if ((zero_any & ((2u << kk) - 1u)) != 0u) {                   // something needed is not there yet: look again
-                        if (*abortp || gtimer() - tstart > kWaitLimitNs) { *abortp = 1; wok = false; break; }
+                        if (abortp->abort || gtimer() - tstart > abortp->limit_ns) { abortp->abort = 1; wok = false; break; }
                         continue;
                     }
                     if (incl_all) { far = d0 + kk; break; }
@@ -282,16 +285,16 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
             if (wok) {
                 const float2 out_state = make_float2(fmaf(a_seg, in.x, tot.x), fmaf(a_seg, in.y, tot.y));
                 if (col_ok) {
-                    st_rec2(my_rec + 2 * lane, kFlagInclusive, out_state);
+                    if (!(p.test_stall && seg == 1)) st_rec2(my_rec + 2 * lane, kFlagInclusive, out_state);
                     if (seg == p.S - 1 && p.state) *reinterpret_cast<float2*>(p.state + (long long)b * p.D + col0 + 2 * lane) = out_state;
                 }
                 if (lane < kNP) *reinterpret_cast<float2*>(&carry[2 * lane]) = in;
             } else if (lane == 0) {
-                *abortp = 1;
+                abortp->abort = 1;
             }
         }
         __syncthreads();
-        if (abort_flag) break;
+        if (wait_ctl.abort) break;
 
         // ---- 3. scan again from the true incoming state and store: sixteen lanes cover one 128-byte row
         {
@@ -332,10 +335,10 @@ __global__ void __launch_bounds__(kSegThreads, kSegCtasPerSm) l2_summary_seg_ker
     }
     // A CTA that gave up may still have a load in flight: wait for it (bounded) before the shared memory goes away.
     __syncthreads();
-    if (tid == 0 && abort_flag) {
+    if (tid == 0 && wait_ctl.abort) {
         if (pending_s >= 0) {
             const unsigned long long tstart = gtimer();
-            while (!mbar_try(&full, (uint32_t)pending_s) && gtimer() - tstart < kWaitLimitNs) {}
+            while (!mbar_try(&full, (uint32_t)pending_s) && gtimer() - tstart < wait_ctl.limit_ns) {}
         }
         if (p.status) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
     }
@@ -388,7 +391,9 @@ cudaError_t launch_l2_summary_seg(const void* X, void* M2, float* state, int use
     p.ticket = static_cast<unsigned int*>(scratch);
     p.rec = reinterpret_cast<unsigned long long*>(static_cast<char*>(scratch) + 256);
     p.M2 = M2; p.state = state; p.T = T; p.n_prev = n_prev; p.B = B; p.D = D; p.kind = kind; p.beta = beta;
-    p.use_state = use_state; p.status = status;
+    p.use_state = use_state; p.status = status; p.wait_limit_ns = wait_limit_ns();
+    p.test_stall = (kind & MKA_SUMMARY_TEST_STALL) ? 1 : 0;
+    kind &= ~MKA_SUMMARY_TEST_STALL;
     if (dtype == MKA_F32) return kind == MKA_SUMMARY_EMA ? launch_k<float, true>(X, p, st) : launch_k<float, false>(X, p, st);
     return kind == MKA_SUMMARY_EMA ? launch_k<__nv_bfloat16, true>(X, p, st) : launch_k<__nv_bfloat16, false>(X, p, st);
 }

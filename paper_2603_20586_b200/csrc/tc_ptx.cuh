@@ -9,7 +9,14 @@
 
 namespace mka {
 
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // every device-side wait gives up after 1 s
+// Every device-side wait gives up after a wall-clock limit: one second unless mka_set_wait_limit_us changed it.
+// The launchers read the limit on the host (wait_limit_ns) and pass it to the kernel, which keeps it in shared memory
+// beside the flag that tells the other roles of the CTA that somebody gave up.
+struct WaitCtl {
+    int abort;                       // set by the first wait that ran out; every other wait of the CTA then returns false
+    unsigned long long limit_ns;
+};
+unsigned long long wait_limit_ns();   // host
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
@@ -33,15 +40,15 @@ __device__ __forceinline__ unsigned long long gtimer() {
     return t;
 }
 // Bounded wait: false when the limit expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile WaitCtl* ctl) {
     if (mbar_try(b, parity)) return true;
     const unsigned long long t0 = gtimer();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 32; ++i)
             if (mbar_try(b, parity)) return true;
-        if (*abort_flag) return false;
-        if (gtimer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+        if (ctl->abort) return false;
+        if (gtimer() - t0 > ctl->limit_ns) { ctl->abort = 1; return false; }
     }
 }
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int x, int y, int z, int w, uint64_t* bar) {
@@ -107,8 +114,8 @@ __device__ __forceinline__ void mma_commit_elect(uint64_t* bar) {
                  ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait executed by every lane of a converged warp; the result is made warp-uniform.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag));
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* b, uint32_t parity, volatile WaitCtl* ctl) {
+    return __all_sync(0xffffffffu, mbar_wait(b, parity, ctl));
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }

@@ -166,3 +166,11 @@ def test_summary_and_paged_workspace_queries(mka):
     assert (ws - 256) % (4 * 28 * 130 * 4) == 0 and 3 <= slots <= sum(-(-x // 128) for x in n)
     # grouped heads in the dense decode take the same split as the paged decode
     assert mka.mka_workspace_bytes(mka.make_shape(4, 28, 1, 128, kv_heads=4), n, b.MKA_WS_DECODE) == ws
+
+
+def test_wait_limit_setter_clamps_and_returns_the_previous_value(mka):
+    old = mka.mka_set_wait_limit_us(5)
+    assert mka.mka_set_wait_limit_us(20_000_000) == 100          # 5 was raised to the floor
+    assert mka.mka_set_wait_limit_us(0) == 10_000_000            # and 20 s lowered to the ceiling
+    assert mka.mka_set_wait_limit_us(old) == 1_000_000           # 0 = the default
+    assert old == 1_000_000

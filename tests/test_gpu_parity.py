@@ -241,9 +241,37 @@ def test_bwd_matches_oracle(mka, orc, case, dtype, flags):
     assert err(g["dG"], ref["dG"])[0] <= tol
     assert abs(float(g["dG"].sum(-1).abs().max())) <= tol            # sum_l dG_l = 0
     dW, db = orc.router_bwd(np64(P["X"]), ref["dG"])
+    # dW_r, db_r are sums over all B*T tokens, so their size grows with the problem: the contract's bound is
+    # applied relative to the largest entry (never below 1)
     scale = max(1.0, float(np.abs(dW).max()))
-    assert err(g["dW_r"], dW)[0] <= (5e-2 if dtype == torch.bfloat16 else 2e-4) * scale
-    assert err(g["db_r"], db)[0] <= (5e-2 if dtype == torch.bfloat16 else 2e-4) * max(1.0, float(np.abs(db).max()))
+    assert err(g["dW_r"], dW)[0] <= tol * scale
+    assert err(g["db_r"], db)[0] <= tol * max(1.0, float(np.abs(db).max()))
+
+
+@pytest.mark.parametrize("zero_slot", [False, True])
+def test_bwd_single_long_term_slot(mka, orc, zero_slot):
+    """One long-term slot (the "Retrieve ∪ {0}" case when it is all zeros, Alg. 1's M3 = 0): every query puts a large
+    share of its mass on that one key, so its dK, dV sum the rounding of all T rows."""
+    B, H, T, d, W, N = 1, 2, 384, 128, 64, (384, 384, 1)
+    P = problem(41, B, H, T, d, N, 32, torch.bfloat16, router_std=0.3, with_dO=True)
+    if zero_slot:
+        P["K"][2].zero_(); P["V"][2].zero_()
+    gate = mka.mka_router(P["X"], P["W_r"], None)
+    shape = mka.make_shape(B, H, T, d, 32, W)
+    assert mka.mka_bwd_kernel_kind(shape, P["K"], P["V"]) == 1
+    O, LSE = mka.mka_fwd(shape, P["Q"], P["K"], P["V"], gate)
+    g = mka.mka_bwd(shape, P["Q"], P["K"], P["V"], gate, O, LSE, P["dO"])
+    rg, _ = orc.router(np64(P["X"]), np64(P["W_r"]))
+    ref = orc.bwd(P["Q"], P["K"], P["V"], rg, P["dO"], W)
+    check(g["dQ"], ref["dQ"], torch.bfloat16, "dQ")
+    for l in range(3):
+        mx, mean = err(g["dK"][l], ref["dK"][l])
+        mxv, meanv = err(g["dV"][l], ref["dV"][l])
+        print(f"single slot (zero={zero_slot}) level {l}: dK max {mx:.3e} mean {mean:.3e}; dV max {mxv:.3e} mean {meanv:.3e}; "
+              f"|dK| max {np.abs(ref['dK'][l]).max():.3e} |dV| max {np.abs(ref['dV'][l]).max():.3e}")
+        check(g["dK"][l], ref["dK"][l], torch.bfloat16, f"dK{l}")
+        check(g["dV"][l], ref["dV"][l], torch.bfloat16, f"dV{l}")
+    assert err(g["dG"], ref["dG"])[0] <= 2e-2
 
 
 @pytest.mark.parametrize("flags", [0, 1])
