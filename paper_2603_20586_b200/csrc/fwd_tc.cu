@@ -29,8 +29,17 @@ namespace mka {
 namespace {
 
 constexpr int kNumQ = 2;
-constexpr int kThreads = 320;
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kSoftmaxWarps = 8 * kNumQ;             // per query tile: two column halves x four lane quarters
+constexpr int kThreads = (kSoftmaxWarps + 4) * 32;    // a fifth warpgroup holds the producer, the issuing warp and two idle warps
+constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
+// Registers are re-divided between the warpgroups at the start of the kernel: the softmax threads keep 64 scores
+// and their weights in registers, the fifth warpgroup needs few.  The kernel is launched with 96 registers per
+// thread (640 threads), and what the five warpgroups hold afterwards must not exceed that pool, or the increase
+// would wait forever: 512 x 104 + 128 x 64 = 640 x 96.
+constexpr int kRegsLaunch = 96, kRegsSoftmax = 104, kRegsOther = 64;
+static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kThreads * kRegsLaunch, "register pool of the CTA exceeded");
+static_assert(kThreads * (kRegsLaunch + 8) > 65536, "the launch would get more than kRegsLaunch registers per thread");
+constexpr int kHalfN = kTileN / 2;                   // key columns of one softmax thread
 constexpr uint32_t kPanelBytes = 128 * 128;          // [128 rows][64 bf16] with 128-byte rows
 constexpr float kRescaleThreshold = 8.0f;            // log2 units
 
@@ -104,6 +113,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     __shared__ Barriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ WaitCtl wait_ctl;
+    __shared__ float xmax[2][kNumQ][2][kTileM];           // row maxima of the two column halves, double-buffered by tile parity
+    __shared__ float lsum[kNumQ][2][kTileM];              // row sums of the two column halves (epilogue)
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
@@ -121,8 +132,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             mbar_init(&bar.v_full[s], 1); mbar_init(&bar.v_empty[s], 1);
         }
         for (int q = 0; q < kNumQ; ++q) {
-            mbar_init(&bar.s_full[q], 1); mbar_init(&bar.p_full[q], kTileM); mbar_init(&bar.pv_done[q], 1);
-            mbar_init(&bar.s_free[q], kTileM);
+            mbar_init(&bar.s_full[q], 1); mbar_init(&bar.p_full[q], 8); mbar_init(&bar.pv_done[q], 1);   // 8 = one arrival per softmax warp
+            mbar_init(&bar.s_free[q], 8);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -155,6 +166,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     }
     const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
 
+    if (warp >= kSoftmaxWarps) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (warp == kProducerWarp && kPaged) {
         // Paged levels: the whole warp produces.  Lane i owns box i of every key tile (a box = the rows of one page
         // that fall into the tile): it looks its page up while the warp waits for the stage to drain and issues its
@@ -292,7 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 }
             }
             auto scrub_v = [&](int e, int s) {
-                if (!kPaged) return;
+                if constexpr (kPaged) {
 #pragma unroll
                 for (int l = 0; l < 3; ++l) {
                     if (e != scrub_e[l]) continue;
@@ -303,6 +316,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
+                }
                 }
             };
             auto issue_pv = [&](int q, int s, bool accumulate) {
@@ -378,30 +392,44 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             }
             }   // !kSeparateP
         }
+    }
     } else {
-        // ------------------------------------------------------------ softmax warpgroups
-        const int q = warp >> 2;
-        const int row_in_tile = tid & (kTileM - 1);
-        const long long t = m0 + (long long)q * kTileM + row_in_tile;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        // ------------------------------------------------------------ softmax warps
+        // Eight warps per query tile: warp = (query tile, column half, lane quarter).  A thread owns 64 key columns of
+        // one query row; the two threads of a row agree on the row maximum through shared memory at a 256-thread
+        // barrier that also carries their "no wait has run out" flags, so that the 256 threads always leave together.
+        const int q = warp >> 3, half = (warp >> 2) & 1;
+        const int row_in_tile = (warp & 3) * 32 + lane;
+        const int t = (int)m0 + q * kTileM + row_in_tile;    // T < 2^31
         const bool row_valid = t < p.T;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t s_addr = tmem + lane_base + q * kTileN;
-        const uint32_t o_addr = tmem + lane_base + 256 + q * DH;
-        const uint32_t p_addr = C::kSeparateP ? tmem + lane_base + C::kColP + q * (kTileN / 2) : s_addr;   // where P (bf16) goes
+        const uint32_t s_addr = tmem + lane_base + q * kTileN + half * kHalfN;
+        const uint32_t o_addr = tmem + lane_base + 256 + q * DH + half * (DH / 2);
+        // where this thread's 64 weights go as 32 bf16 pairs
+        const uint32_t p_addr = (C::kSeparateP ? tmem + lane_base + C::kColP + q * (kTileN / 2) : tmem + lane_base + q * kTileN) + half * (kHalfN / 2);
         const long long tq0 = m0 + (long long)q * kTileM;                      // first row of this query tile
         const long long tq1 = (tq0 + kTileM - 1 < p.T - 1) ? tq0 + kTileM - 1 : p.T - 1;
+        auto pair_all = [&](bool flag) -> bool {                                // AND over the 256 threads of the query tile
+            uint32_t out;
+            asm volatile("{\n.reg .pred pi, po;\nsetp.ne.u32 pi, %1, 0;\nbar.red.and.pred po, %2, 256, pi;\nselp.u32 %0, 1, 0, po;\n}"
+                         : "=r"(out) : "r"((uint32_t)flag), "r"(1 + q) : "memory");
+            return out != 0;
+        };
 
-        float m_run = -INFINITY, l_run = 0.f;
-        bool ok = true;
+        float m_run = -INFINITY, l_run = 0.f;                                    // l_run: this thread's 64 columns only
+        bool ok = true, all_ok = true;                                           // ok is warp-uniform
         int e = 0;
-        for (int l = 0; l < 3 && ok; ++l) {
+        for (int l = 0; l < 3 && all_ok; ++l) {
             if (first[l] == end[l]) continue;
             float bias = -INFINITY;
-            long long lo = 0, hi = 0;
+            int lo = 0, hi = 0;                              // visible rows of this level (levels hold fewer than 2^31 rows)
             if (row_valid) {
                 const float g = p.gate[((long long)b * p.T + t) * 3 + l];
                 bias = g > 0.f ? log2f(g) : -INFINITY;
-                visible_range(l, t + p.q_offset, p.window, nl[l], 0, lo, hi);
+                long long lo64, hi64;
+                visible_range(l, (long long)t + p.q_offset, p.window, nl[l], 0, lo64, hi64);
+                lo = (int)lo64; hi = (int)hi64;
             }
             // key tiles visible to every row of THIS query tile need no element mask
             int full_first = 0, full_end = 0;
@@ -414,29 +442,42 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 if (tq1 - tq0 + 1 < kTileM) full_end = full_first;         // ragged query tile: always mask
             }
             for (int kt = first[l]; kt < end[l]; ++kt, ++e) {
-                ok = mbar_wait(&bar.s_full[q], (uint32_t)e & 1u, abortp);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                tc_fence_after();
-                float s[kTileN];
-#pragma unroll
-                for (int c0 = 0; c0 < kTileN; c0 += 32) tmem_ld32(s_addr + c0, reinterpret_cast<uint32_t*>(s) + c0);
-                tmem_ld_wait();
-                if (C::kSeparateP) {                         // S(e) is in registers: its TMEM columns may be reused
-                    tc_fence_before();
-                    mbar_arrive(&bar.s_free[q]);
-                }
-                const bool need_mask = !(kt >= full_first && kt < full_end);
-                if (need_mask) {
-                    const int c_lo = (int)max(-1LL, min(lo - (long long)kt * kTileN, (long long)kTileN));
-                    const int c_hi = (int)max(-1LL, min(hi - (long long)kt * kTileN, (long long)kTileN));
-#pragma unroll
-                    for (int c = 0; c < kTileN; ++c)
-                        if (c < c_lo || c >= c_hi) s[c] = -INFINITY;
-                }
+                if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bar.s_full[q], (uint32_t)e & 1u, abortp));
+                float s[kHalfN];
                 float mx = -INFINITY;
+                if (ok) {
+                    tc_fence_after();
 #pragma unroll
-                for (int c = 0; c < kTileN; ++c) mx = fmaxf(mx, s[c]);
+                    for (int c0 = 0; c0 < kHalfN; c0 += 32) tmem_ld32(s_addr + c0, reinterpret_cast<uint32_t*>(s) + c0);
+                    tmem_ld_wait();
+                    if (C::kSeparateP) {                     // S(e) is in registers: its TMEM columns may be reused
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bar.s_free[q]);
+                    }
+                    const bool need_mask = !(kt >= full_first && kt < full_end);
+                    if (need_mask) {
+                        const long long col0 = (long long)kt * kTileN + half * kHalfN;
+                        const int c_lo = (int)max(-1LL, min((long long)lo - col0, (long long)kHalfN));
+                        const int c_hi = (int)max(-1LL, min((long long)hi - col0, (long long)kHalfN));
+#pragma unroll
+                        for (int c = 0; c < kHalfN; ++c)
+                            if (c < c_lo || c >= c_hi) s[c] = -INFINITY;
+                    }
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < kHalfN; c += 8) {
+                        mx4[0] = max3(mx4[0], s[c], s[c + 1]); mx4[1] = max3(mx4[1], s[c + 2], s[c + 3]);
+                        mx4[2] = max3(mx4[2], s[c + 4], s[c + 5]); mx4[3] = max3(mx4[3], s[c + 6], s[c + 7]);
+                    }
+                    mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                }
+                // With P written over S (d = 128) this barrier is also what lets a thread overwrite columns that the
+                // other half of its row has read: both halves have their scores in registers when it completes.
+                xmax[e & 1][q][half][row_in_tile] = mx;
+                all_ok = pair_all(ok);
+                if (!all_ok) break;
+                mx = fmaxf(mx, xmax[e & 1][q][half ^ 1][row_in_tile]);
                 const float x_max = fmaf(mx, p.scale_log2, bias);            // -inf when the whole row is masked
                 const float m_new = fmaxf(m_run, x_max);
                 const bool grow = m_new > m_run + kRescaleThreshold;         // also true for the first finite max
@@ -444,57 +485,64 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 const float m_eff = m_use == -INFINITY ? 0.f : m_use;
                 const float alpha = grow ? (m_run == -INFINITY ? 0.f : ex2(m_run - m_use)) : 1.f;
                 const float shift = bias - m_eff;
-                float sum = 0.f;
-                uint32_t pk[kTileN / 2];
-#pragma unroll
-                for (int c = 0; c < kTileN; c += 2) {
-                    const float p0 = ex2(fmaf(s[c], p.scale_log2, shift));
-                    const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, shift));
-                    sum += p0 + p1;
-                    pk[c / 2] = pack_bf16(p0, p1);
-                }
-                l_run = fmaf(l_run, alpha, sum);
+                l_run *= alpha;
                 m_run = m_use;
-                if (C::kSeparateP && e > 0) {                // P(e-1) must have been consumed before P(e) replaces it
-                    ok = mbar_wait(&bar.pv_done[q], (uint32_t)(e - 1) & 1u, abortp);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
+                // P(e-1) must have been consumed before P(e) replaces it (d = 64), and before O is rescaled
+                const bool rescale = e > 0 && __any_sync(0xffffffffu, alpha != 1.f);
+                if ((C::kSeparateP || rescale) && e > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bar.pv_done[q], (uint32_t)(e - 1) & 1u, abortp));
+                    if (ok) tc_fence_after();
                 }
-                tmem_st32(p_addr, pk);
-                tmem_st32(p_addr + 32, pk + 32);
-                // O accumulator rescale (only when some row of this warp moved its reference maximum)
-                if (e > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                    ok = mbar_wait(&bar.pv_done[q], (uint32_t)(e - 1) & 1u, abortp);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
+                if (ok) {
+                    float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                    for (int c0 = 0; c0 < DH; c0 += 32) {
-                        uint32_t o[32];
-                        tmem_ld32(o_addr + c0, o);
-                        tmem_ld_wait();
+                    for (int c0 = 0; c0 < kHalfN; c0 += 32) {           // 32 columns = 16 packed pairs per store
+                        uint32_t pk[16];
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(o_addr + c0, o);
+                        for (int c = c0; c < c0 + 32; c += 4) {
+                            const float p0 = ex2(fmaf(s[c], p.scale_log2, shift));
+                            const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, shift));
+                            const float p2 = ex2(fmaf(s[c + 2], p.scale_log2, shift));
+                            const float p3 = ex2(fmaf(s[c + 3], p.scale_log2, shift));
+                            sum0 += p0 + p1;
+                            sum1 += p2 + p3;
+                            pk[(c - c0) / 2] = pack_bf16(p0, p1);
+                            pk[(c - c0) / 2 + 1] = pack_bf16(p2, p3);
+                        }
+                        tmem_st16(p_addr + c0 / 2, pk);
                     }
+                    l_run += sum0 + sum1;
+                    if (rescale) {                           // some row of this warp moved its reference maximum
+#pragma unroll 1
+                        for (int c0 = 0; c0 < DH / 2; c0 += 32) {
+                            uint32_t o[32];
+                            tmem_ld32(o_addr + c0, o);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(o_addr + c0, o);
+                        }
+                    }
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bar.p_full[q]);
                 }
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(&bar.p_full[q]);
             }
         }
         // ------------------------------------------------------------ epilogue
-        __nv_bfloat16* Orow = p.O + (((long long)b * p.H + h) * p.T + t) * DH;
-        if (ok && E > 0) {
-            ok = mbar_wait(&bar.pv_done[q], (uint32_t)(E - 1) & 1u, abortp);
-            ok = __all_sync(0xffffffffu, ok);
+        if (all_ok) {
+            if (ok && E > 0) ok = __all_sync(0xffffffffu, mbar_wait(&bar.pv_done[q], (uint32_t)(E - 1) & 1u, abortp));
+            lsum[q][half][row_in_tile] = l_run;              // the row's sum is the sum of its two halves
+            all_ok = pair_all(ok);
         }
-        if (ok) {
+        if (all_ok) {
             tc_fence_after();
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-#pragma unroll
-            for (int c0 = 0; c0 < DH; c0 += 32) {
+            const float l_row = l_run + lsum[q][half ^ 1][row_in_tile];
+            const float inv = l_row > 0.f ? 1.f / l_row : 0.f;   // rows with nothing visible: exact zeros
+            __nv_bfloat16* Orow = p.O + (((long long)b * p.H + h) * p.T + t) * DH + half * (DH / 2);
+#pragma unroll 1
+            for (int c0 = 0; c0 < DH / 2; c0 += 32) {
                 uint32_t o[32];
                 if (E > 0) {
                     tmem_ld32(o_addr + c0, o);
@@ -507,7 +555,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         uint4 v;
-                        const float z = inv;   // rows with nothing visible: inv = 0 -> exact zeros
+                        const float z = inv;
                         v.x = pack_bf16(z > 0.f ? __uint_as_float(o[i]) * z : 0.f, z > 0.f ? __uint_as_float(o[i + 1]) * z : 0.f);
                         v.y = pack_bf16(z > 0.f ? __uint_as_float(o[i + 2]) * z : 0.f, z > 0.f ? __uint_as_float(o[i + 3]) * z : 0.f);
                         v.z = pack_bf16(z > 0.f ? __uint_as_float(o[i + 4]) * z : 0.f, z > 0.f ? __uint_as_float(o[i + 5]) * z : 0.f);
@@ -516,8 +564,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     }
                 }
             }
-            if (row_valid && p.LSE)
-                p.LSE[((long long)b * p.H + h) * p.T + t] = l_run > 0.f ? (m_run + log2f(l_run)) * kLn2 : -INFINITY;
+            if (row_valid && half == 0 && p.LSE)
+                p.LSE[((long long)b * p.H + h) * p.T + t] = l_row > 0.f ? (m_run + log2f(l_row)) * kLn2 : -INFINITY;
         }
     }
 
