@@ -1,26 +1,33 @@
 // Tensor-core forward of Eq. 5 for bf16 on sm_100a: TMA -> shared memory -> tcgen05.mma -> TMEM.
 //
-// One CTA owns 256 query rows (two 128-row tiles, "ping" and "pong") of one (batch, head) and walks
-// ONE level-ordered list of 128-row key tiles: all visible L1 tiles, then L2, then L3.  A single
-// running (max, sum) per row spans the three levels (the max shift of Eq. 11-14); the gate enters
-// as a per-row, per-level additive bias log2(lambda) inside the exponent, so that
+// A CTA owns 128-row query tiles of one (batch, head) -- two of them ("ping" and "pong", 256 rows) at d = 128, one at
+// d = 64, where two CTAs share an SM -- and walks ONE level-ordered list of 128-row key tiles: all visible L1 tiles,
+// then L2, then L3.  A single running (max, sum) per row spans the three levels (the max shift of Eq. 11-14); the gate
+// enters as a per-row, per-level additive bias log2(lambda) inside the exponent, so that
 //     p = 2^(s * tau * log2(e) + log2(lambda_l) - m)  =  lambda_l * exp(s*tau - m')
 // which is exactly the gated, un-normalised weight of Eq. 5.  One normalisation at the end.
 //
-// Warp roles (320 threads):
-//   warps 0-3 / 4-7  softmax warpgroup of query tile 0 / 1: thread i <-> TMEM lane i <-> query row i.
-//                    Reads S from TMEM, applies bias and masks, running max, exp2, writes P (bf16)
-//                    back into the TMEM columns S occupied, rescales the O accumulator when the
-//                    running maximum grows by more than 2^8 (lazy rescale), and does the epilogue.
-//   warp 8           producer: one lane issues the TMA loads of Q and of the K / V tile list into
-//                    128-byte-swizzled shared-memory rings (one mbarrier pair per stage).
-//   warp 9           issues every tcgen05.mma (the warp runs its loop converged, one elected lane issues): S_q = Q_q K^T (both operands from shared
-//                    memory) and O_q += P_q V (P from TMEM, V from shared memory, N-major), in the
-//                    order  S0(e)  O1(e-1)  S1(e)  O0(e)  so that each warpgroup's softmax overlaps
-//                    the other tile's matrix products.
-// TMEM: columns [0,128) S0/P0, [128,256) S1/P1, [256,256+d) O0, [256+d,256+2d) O1.  With d = 64 the 128 columns
-// left over hold P0 and P1 on their own ([384,448), [448,512)), and S_q(e+1) is multiplied while the softmax of
-// S_q(e) runs (the hand-off is "S is in registers", not "P has been consumed").
+// Warp roles (d = 128: 640 threads, d = 64: 384 threads):
+//   8 warps per query tile   softmax: warp = (query tile, column half, lane quarter); a thread owns 64 key columns of
+//                    one query row (TMEM lane = row).  Reads S from TMEM, applies bias and masks, agrees with the
+//                    row's other thread on the maximum (shared memory + a 256-thread barrier), exp2, packs the
+//                    weights to bf16 and writes them to TMEM in two parts of 32 keys (at d = 128 over the columns S
+//                    occupied), rescales the O accumulator when the running maximum grows by more than 2^8 (lazy
+//                    rescale), and does the epilogue for its half of the row.
+//   next warp        producer: one lane issues the TMA loads of Q and of the K / V tile list into 128-byte-swizzled
+//                    shared-memory rings (one mbarrier pair per stage); with paged levels the whole warp produces.
+//   next warp        issues every tcgen05.mma (the warp runs its loop converged, one elected lane issues):
+//                    S_q = Q_q K^T (both operands from shared memory) and O_q += P_q V (P from TMEM, V from shared
+//                    memory, N-major) in two halves that follow the two parts of P, so that the first half runs under
+//                    the remaining exponentials.  At d = 128 the order is  S0(e)  O1(e-1)  S1(e)  O0(e):  each tile's
+//                    softmax overlaps the other tile's products.
+//   two idle warps   complete the last warpgroup, so that registers can be moved between warpgroups (setmaxnreg).
+// TMEM: S tiles first (128 columns each), then the O accumulators (d columns each); at d = 64 a P region of 64 columns
+// per query tile follows, and S_q(e+1) is multiplied while the softmax of S_q(e) runs (the hand-off is "S is in
+// registers", not "P has been consumed").  d = 128 uses all 512 columns, d = 64 256.
+// What bounds the d = 128 kernel is the chain  softmax_q(e) -> O_q += P V -> S_q(e+1) -> softmax_q(e+1):  a key tile
+// costs the tensor pipe 2048 cycles and the special-function unit 2048 cycles for the two query tiles, but S_q(e+1)
+// cannot be written before P_q(e), which lies over S_q(e), has been consumed, and TMEM has no room for a second S.
 // Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA raises a flag in shared
 // memory, writes the device status word, lets every role drain, frees TMEM and returns.
 #include "tc_ptx.cuh"
@@ -28,17 +35,6 @@
 namespace mka {
 namespace {
 
-constexpr int kNumQ = 2;
-constexpr int kSoftmaxWarps = 8 * kNumQ;             // per query tile: two column halves x four lane quarters
-constexpr int kThreads = (kSoftmaxWarps + 4) * 32;    // a fifth warpgroup holds the producer, the issuing warp and two idle warps
-constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
-// Registers are re-divided between the warpgroups at the start of the kernel: the softmax threads keep 64 scores
-// and their weights in registers, the fifth warpgroup needs few.  The kernel is launched with 96 registers per
-// thread (640 threads), and what the five warpgroups hold afterwards must not exceed that pool, or the increase
-// would wait forever: 512 x 104 + 128 x 64 = 640 x 96.
-constexpr int kRegsLaunch = 96, kRegsSoftmax = 104, kRegsOther = 64;
-static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kThreads * kRegsLaunch, "register pool of the CTA exceeded");
-static_assert(kThreads * (kRegsLaunch + 8) > 65536, "the launch would get more than kRegsLaunch registers per thread");
 constexpr int kHalfN = kTileN / 2;                   // key columns of one softmax thread
 constexpr uint32_t kPanelBytes = 128 * 128;          // [128 rows][64 bf16] with 128-byte rows
 constexpr float kRescaleThreshold = 8.0f;            // log2 units
@@ -71,23 +67,44 @@ struct TcParams {
 
 template <int DH>
 struct Cfg {
+    // d = 128: one CTA per SM with two query tiles (all 512 TMEM columns).  d = 64: the scores of one key tile cost the
+    // special-function unit as much as at d = 128 but only half the tensor work, and the tile lists of the training
+    // shapes are short; there a CTA takes ONE query tile (256 TMEM columns) and two CTAs share the SM, so that one CTA's
+    // start-up, waits and epilogue run under the other's steady state.
+    static constexpr int kNumQ = DH == 128 ? 2 : 1;
+    static constexpr int kCtasPerSm = DH == 128 ? 1 : 2;
+    static constexpr int kSoftmaxWarps = 8 * kNumQ;         // per query tile: two column halves x four lane quarters
+    static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;   // one more warpgroup: the producer, the issuing warp, two idle warps
+    static constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
+    // Registers are re-divided between the warpgroups at the start of the kernel: the softmax threads keep 64 scores
+    // and their weights in registers, the last warpgroup needs few.  What the warpgroups hold afterwards must not exceed
+    // what the launch gave the CTA, or the increase would wait forever:
+    //   d = 128: 640 threads x 96 at launch = 512 x 104 + 128 x 64;   d = 64: 384 x 80 = 256 x 104 + 128 x 32.
+    static constexpr int kRegsLaunch = DH == 128 ? 96 : 80, kRegsSoftmax = 104, kRegsOther = DH == 128 ? 64 : 32;
+    static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kThreads * kRegsLaunch, "register pool of the CTA exceeded");
+    static_assert(kThreads * kCtasPerSm * (kRegsLaunch + 8) > 65536, "the launch would get more than kRegsLaunch registers per thread");
     static constexpr int kPanels = DH / 64;
     static constexpr uint32_t kTileBytes = kPanels * kPanelBytes;
-    static constexpr int kStages = DH == 128 ? 2 : 4;
+    static constexpr int kStages = 2;
     static constexpr uint32_t kSmemBytes = (kNumQ + 2 * kStages) * kTileBytes + 1024;
     static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-    // With d = 64 the two O accumulators leave 128 TMEM columns free: P gets a region of its own there instead of
+    // With d = 64 the O accumulator leaves TMEM columns free: P gets a region of its own there instead of
     // overwriting S, so S(e+1) can be multiplied while the softmax of S(e) is still running.
     static constexpr bool kSeparateP = DH == 64;
-    static constexpr uint32_t kColP = 256 + kNumQ * DH;       // first P column when kSeparateP
+    static constexpr uint32_t kColO = kNumQ * kTileN;          // first accumulator column (S tiles come first)
+    static constexpr uint32_t kColP = kColO + kNumQ * DH;     // first P column when kSeparateP
+    static constexpr uint32_t kTmemCols = DH == 128 ? 512u : 256u;
+    static_assert(kColP + (kSeparateP ? kNumQ * (kTileN / 2) : 0) <= kTmemCols, "TMEM columns exceeded");
     static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 };
+
+constexpr int kMaxQ = 2;
 
 struct Barriers {
     uint64_t q_full;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[kNumQ], p_full[kNumQ], pv_done[kNumQ];
-    uint64_t s_free[kNumQ];   // d = 64 only: the warpgroup has read S(e) into registers, S(e+1) may overwrite it
+    uint64_t s_full[kMaxQ], p_part[kMaxQ][2], pv_done[kMaxQ];   // p_part: the first / second 32 keys of both column halves are written
+    uint64_t s_free[kMaxQ];   // d = 64 only: the warpgroup has read S(e) into registers, S(e+1) may overwrite it
 };
 
 // Key-tile range [first, end) of a block of query rows [r0, r1] (inclusive) on one level.
@@ -103,25 +120,25 @@ __device__ __forceinline__ void tile_range(int level, long long r0, long long r1
 }
 
 template <int DH, bool kPaged>
-__global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+__global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     using C = Cfg<DH>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint8_t* sQ = smem;                                   // kNumQ tiles
-    uint8_t* sK = sQ + kNumQ * C::kTileBytes;             // kStages tiles
+    uint8_t* sQ = smem;                                   // C::kNumQ tiles
+    uint8_t* sK = sQ + C::kNumQ * C::kTileBytes;             // kStages tiles
     uint8_t* sV = sK + C::kStages * C::kTileBytes;        // kStages tiles
     __shared__ Barriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ WaitCtl wait_ctl;
-    __shared__ float xmax[2][kNumQ][2][kTileM];           // row maxima of the two column halves, double-buffered by tile parity
-    __shared__ float lsum[kNumQ][2][kTileM];              // row sums of the two column halves (epilogue)
+    __shared__ float xmax[2][C::kNumQ][2][kTileM];           // row maxima of the two column halves, double-buffered by tile parity
+    __shared__ float lsum[C::kNumQ][2][kTileM];              // row sums of the two column halves (epilogue)
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
     const int b = blockIdx.z, h = blockIdx.y;
     const int qpair = gridDim.x - 1 - blockIdx.x;          // heaviest (latest) rows first
-    const long long m0 = (long long)qpair * (kNumQ * kTileM);
-    const long long m_last = (m0 + kNumQ * kTileM - 1 < p.T - 1) ? m0 + kNumQ * kTileM - 1 : p.T - 1;
+    const long long m0 = (long long)qpair * (C::kNumQ * kTileM);
+    const long long m_last = (m0 + C::kNumQ * kTileM - 1 < p.T - 1) ? m0 + C::kNumQ * kTileM - 1 : p.T - 1;
 
     if (tid == 0) {
         wait_ctl.abort = 0;
@@ -131,14 +148,15 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             mbar_init(&bar.k_full[s], 1); mbar_init(&bar.k_empty[s], 1);
             mbar_init(&bar.v_full[s], 1); mbar_init(&bar.v_empty[s], 1);
         }
-        for (int q = 0; q < kNumQ; ++q) {
-            mbar_init(&bar.s_full[q], 1); mbar_init(&bar.p_full[q], 8); mbar_init(&bar.pv_done[q], 1);   // 8 = one arrival per softmax warp
+        for (int q = 0; q < C::kNumQ; ++q) {
+            mbar_init(&bar.s_full[q], 1); mbar_init(&bar.pv_done[q], 1);
+            mbar_init(&bar.p_part[q][0], 8); mbar_init(&bar.p_part[q][1], 8);   // 8 = one arrival per softmax warp
             mbar_init(&bar.s_free[q], 8);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(C::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -166,16 +184,16 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     }
     const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
 
-    if (warp >= kSoftmaxWarps) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
-    if (warp == kProducerWarp && kPaged) {
+    if (warp >= C::kSoftmaxWarps) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
+    if (warp == C::kProducerWarp && kPaged) {
         // Paged levels: the whole warp produces.  Lane i owns box i of every key tile (a box = the rows of one page
         // that fall into the tile): it looks its page up while the warp waits for the stage to drain and issues its
         // own copies, so a tile costs one table round trip (overlapped) and four warp-wide copy instructions.
         if (lane == 0) {
-            mbar_expect_tx(&bar.q_full, kNumQ * C::kTileBytes);
+            mbar_expect_tx(&bar.q_full, C::kNumQ * C::kTileBytes);
 #pragma unroll
-            for (int q = 0; q < kNumQ; ++q)
+            for (int q = 0; q < C::kNumQ; ++q)
 #pragma unroll
                 for (int pn = 0; pn < C::kPanels; ++pn)
                     tma_load_4d(sQ + q * C::kTileBytes + pn * kPanelBytes, &maps.q, pn * 64, (int)(m0 + q * kTileM), h, b, &bar.q_full);
@@ -230,11 +248,11 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             mbar_wait_warp(&bar.k_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
             mbar_wait_warp(&bar.v_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
-    } else if (warp == kProducerWarp) {
+    } else if (warp == C::kProducerWarp) {
         if (lane == 0) {
-            mbar_expect_tx(&bar.q_full, kNumQ * C::kTileBytes);
+            mbar_expect_tx(&bar.q_full, C::kNumQ * C::kTileBytes);
 #pragma unroll
-            for (int q = 0; q < kNumQ; ++q)
+            for (int q = 0; q < C::kNumQ; ++q)
 #pragma unroll
                 for (int pn = 0; pn < C::kPanels; ++pn)
                     tma_load_4d(sQ + q * C::kTileBytes + pn * kPanelBytes, &maps.q, pn * 64, (int)(m0 + q * kTileM), h, b, &bar.q_full);
@@ -269,7 +287,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
             for (int i = issued_v > C::kStages ? issued_v - C::kStages : 0; i < issued_v; ++i)
                 mbar_wait(&bar.v_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
-    } else if (warp == kMmaWarp) {
+    } else if (warp == C::kMmaWarp) {
         {   // every lane runs the issue loop (converged); elect.sync inside the wrappers picks the issuing lane
             bool ok = mbar_wait_warp(&bar.q_full, 0, abortp);
             tc_fence_after();
@@ -319,13 +337,25 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                 }
                 }
             };
-            auto issue_pv = [&](int q, int s, bool accumulate) {
+            // O_q += P_q V in two parts: the softmax warps hand over the weights of keys {0-31, 64-95} of the tile (K-steps
+            // 0, 1, 4, 5) before they have finished those of keys {32-63, 96-127} (K-steps 2, 3, 6, 7), so the first half
+            // of the product runs under the remaining exponentials.
+            auto issue_pv = [&](int q, int s, int e, bool accumulate) -> bool {
                 const uint32_t va = v_lo + s * (C::kTileBytes >> 4);
+                const uint32_t pa = tmem + (C::kSeparateP ? C::kColP + q * (kTileN / 2) : q * kTileN);
 #pragma unroll
-                for (int k = 0; k < kTileN / 16; ++k)
-                    mma_ts_elect(tmem + 256 + q * DH, tmem + (C::kSeparateP ? C::kColP + q * (kTileN / 2) : q * kTileN) + k * 8,
-                                 make_desc(va + k * (2048 >> 4)), C::kIdescPV, (accumulate || k > 0) ? 1u : 0u);
+                for (int part = 0; part < 2; ++part) {
+                    if (!mbar_wait_warp(&bar.p_part[q][part], (uint32_t)e & 1u, abortp)) return false;
+                    tc_fence_after();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = (i >> 1) * 4 + part * 2 + (i & 1);
+                        mma_ts_elect(tmem + C::kColO + q * DH, pa + k * 8, make_desc(va + k * (2048 >> 4)), C::kIdescPV,
+                                     (accumulate || part > 0 || i > 0) ? 1u : 0u);
+                    }
+                }
                 mma_commit_elect(&bar.pv_done[q]);
+                return true;
             };
             if (C::kSeparateP) {
                 // S_q(e+1) is issued as soon as the warpgroup has S_q(e) in registers; O_q += P_q(e) V(e) when P_q(e) is written.
@@ -341,7 +371,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     if (e + 1 < E) {
                         if (!mbar_wait_warp(&bar.k_full[sn], (uint32_t)((e + 1) / C::kStages) & 1u, abortp)) { ok = false; break; }
 #pragma unroll
-                        for (int q = 0; q < kNumQ; ++q) {
+                        for (int q = 0; q < C::kNumQ; ++q) {
                             if (!mbar_wait_warp(&bar.s_free[q], (uint32_t)e & 1u, abortp)) { ok = false; break; }
                             tc_fence_after();
                             issue_qk(q, sn);
@@ -352,49 +382,42 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     if (!mbar_wait_warp(&bar.v_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) { ok = false; break; }
                     scrub_v(e, s);
 #pragma unroll
-                    for (int q = 0; q < kNumQ; ++q) {
-                        if (!mbar_wait_warp(&bar.p_full[q], (uint32_t)e & 1u, abortp)) { ok = false; break; }
-                        tc_fence_after();
-                        issue_pv(q, s, e > 0);
+                    for (int q = 0; q < C::kNumQ; ++q) {
+                        if (!issue_pv(q, s, e, e > 0)) { ok = false; break; }
                     }
                     if (!ok) break;
                     mma_commit_elect(&bar.v_empty[s]);
                 }
             } else {
+            // The wait for K(e+1) is taken before the wait for P_0(e), so that S_0(e+1) follows O_0(e) at once: that
+            // pair of products is what query tile 0's softmax threads are waiting for.
+            if (ok && E > 0) ok = mbar_wait_warp(&bar.k_full[0], 0, abortp);
             for (int e = 0; e < E && ok; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
-                if (!mbar_wait_warp(&bar.k_full[s], ph, abortp)) { ok = false; break; }
                 tc_fence_after();
                 issue_qk(0, s);
                 if (e > 0) {
                     const int sp = (e - 1) % C::kStages;
-                    if (!mbar_wait_warp(&bar.p_full[1], (uint32_t)(e - 1) & 1u, abortp)) { ok = false; break; }
-                    tc_fence_after();
-                    issue_pv(1, sp, e - 1 > 0);
+                    if (!issue_pv(1, sp, e - 1, e - 1 > 0)) { ok = false; break; }
                     mma_commit_elect(&bar.v_empty[sp]);
                 }
                 issue_qk(1, s);
                 mma_commit_elect(&bar.k_empty[s]);
                 if (!mbar_wait_warp(&bar.v_full[s], ph, abortp)) { ok = false; break; }
                 scrub_v(e, s);
-                if (!mbar_wait_warp(&bar.p_full[0], (uint32_t)e & 1u, abortp)) { ok = false; break; }
-                tc_fence_after();
-                issue_pv(0, s, e > 0);
+                if (e + 1 < E && !mbar_wait_warp(&bar.k_full[(e + 1) % C::kStages], (uint32_t)((e + 1) / C::kStages) & 1u, abortp)) { ok = false; break; }
+                if (!issue_pv(0, s, e, e > 0)) { ok = false; break; }
             }
             if (ok && E > 0) {
                 const int sp = (E - 1) % C::kStages;
-                if (mbar_wait_warp(&bar.p_full[1], (uint32_t)(E - 1) & 1u, abortp)) {
-                    tc_fence_after();
-                    issue_pv(1, sp, E - 1 > 0);
-                    mma_commit_elect(&bar.v_empty[sp]);
-                }
+                if (issue_pv(1, sp, E - 1, E - 1 > 0)) mma_commit_elect(&bar.v_empty[sp]);
             }
             }   // !kSeparateP
         }
     }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
         // ------------------------------------------------------------ softmax warps
         // Eight warps per query tile: warp = (query tile, column half, lane quarter).  A thread owns 64 key columns of
         // one query row; the two threads of a row agree on the row maximum through shared memory at a 256-thread
@@ -405,7 +428,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const bool row_valid = t < p.T;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t s_addr = tmem + lane_base + q * kTileN + half * kHalfN;
-        const uint32_t o_addr = tmem + lane_base + 256 + q * DH + half * (DH / 2);
+        const uint32_t o_addr = tmem + lane_base + C::kColO + q * DH + half * (DH / 2);
         // where this thread's 64 weights go as 32 bf16 pairs
         const uint32_t p_addr = (C::kSeparateP ? tmem + lane_base + C::kColP + q * (kTileN / 2) : tmem + lane_base + q * kTileN) + half * (kHalfN / 2);
         const long long tq0 = m0 + (long long)q * kTileM;                      // first row of this query tile
@@ -494,24 +517,6 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                     if (ok) tc_fence_after();
                 }
                 if (ok) {
-                    float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-                    for (int c0 = 0; c0 < kHalfN; c0 += 32) {           // 32 columns = 16 packed pairs per store
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int c = c0; c < c0 + 32; c += 4) {
-                            const float p0 = ex2(fmaf(s[c], p.scale_log2, shift));
-                            const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, shift));
-                            const float p2 = ex2(fmaf(s[c + 2], p.scale_log2, shift));
-                            const float p3 = ex2(fmaf(s[c + 3], p.scale_log2, shift));
-                            sum0 += p0 + p1;
-                            sum1 += p2 + p3;
-                            pk[(c - c0) / 2] = pack_bf16(p0, p1);
-                            pk[(c - c0) / 2 + 1] = pack_bf16(p2, p3);
-                        }
-                        tmem_st16(p_addr + c0 / 2, pk);
-                    }
-                    l_run += sum0 + sum1;
                     if (rescale) {                           // some row of this warp moved its reference maximum
 #pragma unroll 1
                         for (int c0 = 0; c0 < DH / 2; c0 += 32) {
@@ -523,10 +528,43 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
                             tmem_st32(o_addr + c0, o);
                         }
                     }
+                    // 64 weights in two parts of 32 (16 packed pairs, one store each).  The first part is handed over
+                    // in the middle of the second part's exponentials, when its store has long completed.
+                    // scale, shift and the row sum work on packed pairs: one instruction for two columns
+                    const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), shift2 = pack2(shift, shift);
+                    uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
+                    uint32_t pk[16];
+                    auto weights = [&](int c_from, int c_to, int c_base) {
+#pragma unroll
+                        for (int c = c_from; c < c_to; c += 4) {
+                            float x0, x1, x2, x3;
+                            unpack2(fma2(pack2(s[c], s[c + 1]), scale2, shift2), x0, x1);
+                            unpack2(fma2(pack2(s[c + 2], s[c + 3]), scale2, shift2), x2, x3);
+                            const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                            sum_a = add2(sum_a, pack2(p0, p1));
+                            sum_b = add2(sum_b, pack2(p2, p3));
+                            pk[(c - c_base) / 2] = pack_bf16(p0, p1);
+                            pk[(c - c_base) / 2 + 1] = pack_bf16(p2, p3);
+                        }
+                    };
+                    weights(0, 32, 0);
+                    tmem_st16(p_addr, pk);
+                    weights(32, 48, 32);
+                    tmem_st_wait();                          // the first part (and a rescaled accumulator) is in TMEM
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bar.p_part[q][0]);
+                    weights(48, 64, 32);
+                    tmem_st16(p_addr + 16, pk);
+                    {
+                        float a0, a1;
+                        unpack2(add2(sum_a, sum_b), a0, a1);
+                        l_run += a0 + a1;
+                    }
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bar.p_full[q]);
+                    if (lane == 0) mbar_arrive(&bar.p_part[q][1]);
                 }
             }
         }
@@ -572,7 +610,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (tid == 0 && wait_ctl.abort) atomicExch(p.status, (unsigned int)MKA_ERR_TIMEOUT);
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
 }
 
 inline bool make_map(CUtensorMap* map, const void* base, int d, long long rows, int H, int B, long long sn, long long sh, long long sb) {
@@ -618,8 +656,8 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
     auto kern = fp.paged ? fwd_tc_kernel<DH, true> : fwd_tc_kernel<DH, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<DH>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    dim3 grid((fp.T + kNumQ * kTileM - 1) / (kNumQ * kTileM), fp.H, fp.B);
-    kern<<<grid, kThreads, Cfg<DH>::kSmemBytes, st>>>(maps, p);
+    dim3 grid((fp.T + Cfg<DH>::kNumQ * kTileM - 1) / (Cfg<DH>::kNumQ * kTileM), fp.H, fp.B);
+    kern<<<grid, Cfg<DH>::kThreads, Cfg<DH>::kSmemBytes, st>>>(maps, p);
     return cudaGetLastError();
 }
 
