@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
             mbar_init(&bar.b_full[s], 1); mbar_init(&bar.b_empty[s], 1);
         }
         mbar_init(&bar.s_full[0], 1); mbar_init(&bar.s_full[1], 1);
-        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 256); mbar_init(&bar.ds_full, 256);
+        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 8); mbar_init(&bar.ds_full, 8);   // 8 = one arrival per element-wise warp
         mbar_init(&bar.acc_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -344,8 +344,10 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 full_end = (int)(hi_f / kBlk);
                 if (m_last - m0 + 1 < kBlk) full_end = full_first;          // ragged query tile: always mask
             }
-            float a0 = 0.f, a1 = 0.f, z0 = 0.f, z1 = 0.f;
+            // sums over this thread's columns as packed pairs (even, odd column)
+            uint64_t a2 = pack2(0.f, 0.f), z2 = a2;
             const float bl = bias[l];
+            const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), bl2 = pack2(bl, bl), negD2 = pack2(-Dt, -Dt);
             for (int kt = first[l]; kt < end[l]; ++kt, ++e) {
                 // phase 1: p = 2^(s * scale + bias) for this thread's 64 columns (needs S only)
                 ok = mbar_wait(&bar.s_full[e & 1], (uint32_t)(e >> 1) & 1u, abortp);
@@ -369,10 +371,11 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 }
 #pragma unroll
                 for (int c = 0; c < 64; c += 2) {
-                    pr[c] = ex2(fmaf(pr[c], p.scale_log2, bl));
-                    pr[c + 1] = ex2(fmaf(pr[c + 1], p.scale_log2, bl));
-                    z0 += pr[c];
-                    z1 += pr[c + 1];
+                    float x0, x1;
+                    unpack2(fma2(pack2(pr[c], pr[c + 1]), scale2, bl2), x0, x1);
+                    pr[c] = ex2(x0);
+                    pr[c + 1] = ex2(x1);
+                    z2 = add2(z2, pack2(pr[c], pr[c + 1]));
                 }
                 // phase 2: dS = p (dP - D), written (bf16) over the dP columns just read
                 ok = mbar_wait(&bar.dp_full, (uint32_t)e & 1u, abortp);
@@ -386,17 +389,25 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 uint32_t pk[32];
 #pragma unroll
                 for (int c = 0; c < 64; c += 2) {
-                    a0 = fmaf(pr[c], dp[c], a0);
-                    a1 = fmaf(pr[c + 1], dp[c + 1], a1);
-                    pk[c / 2] = pack_bf16(pr[c] * (dp[c] - Dt), pr[c + 1] * (dp[c + 1] - Dt));
+                    const uint64_t p2 = pack2(pr[c], pr[c + 1]), d2 = pack2(dp[c], dp[c + 1]);
+                    a2 = fma2(p2, d2, a2);
+                    float s0, s1;
+                    unpack2(mul2(p2, add2(d2, negD2)), s0, s1);
+                    pk[c / 2] = pack_bf16(s0, s1);
                 }
                 tmem_st32(dp_addr, pk);
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(&bar.ds_full);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar.ds_full);
             }
-            Al[l] = a0 + a1;
-            Sl[l] = z0 + z1;
+            {
+                float a0, a1, z0, z1;
+                unpack2(a2, a0, a1);
+                unpack2(z2, z0, z1);
+                Al[l] = a0 + a1;
+                Sl[l] = z0 + z1;
+            }
         }
         // ------------------------------------------------------------ epilogue
         if (ok && E > 0) {
@@ -491,7 +502,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
         mbar_init(&bar.fixed_full, 1);
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1); }
         mbar_init(&bar.s_full[0], 1);
-        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 256); mbar_init(&bar.ds_full, 256);
+        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 8); mbar_init(&bar.ds_full, 8);   // 8 = one arrival per element-wise warp
         mbar_init(&bar.acc_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -645,9 +656,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                     if (c < c_lo || c >= c_hi) pr[c] = -INFINITY;
             }
             uint32_t pk[32];        // P^T rounded to bf16; phase 2 uses these same rounded values
+            const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
 #pragma unroll
-            for (int c = 0; c < 64; c += 2)
-                pk[c / 2] = pack_bf16(ex2(fmaf(pr[c], p.scale_log2, st[c])), ex2(fmaf(pr[c + 1], p.scale_log2, st[c + 1])));
+            for (int c = 0; c < 64; c += 2) {
+                float x0, x1;
+                unpack2(fma2(pack2(pr[c], pr[c + 1]), scale2, pack2(st[c], st[c + 1])), x0, x1);
+                pk[c / 2] = pack_bf16(ex2(x0), ex2(x1));
+            }
             tmem_st32(s_addr, pk);
             // D_t of the 64 queries, again ahead of the wait
 #pragma unroll
@@ -657,7 +672,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             }
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(&bar.p_full);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar.p_full);
             // phase 2: dS^T = P^T (dP^T - D_t), written over the dP^T columns just read
             ok = mbar_wait(&bar.dp_full, (uint32_t)e & 1u, abortp);
             ok = __all_sync(0xffffffffu, ok);
@@ -666,15 +682,19 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             tmem_ld32(dp_addr, reinterpret_cast<uint32_t*>(pr));
             tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(pr) + 32);
             tmem_ld_wait();
+            const uint64_t minus1 = pack2(-1.f, -1.f);
 #pragma unroll
             for (int c = 0; c < 64; c += 2) {
                 const float p0 = __uint_as_float(pk[c / 2] << 16), p1 = __uint_as_float(pk[c / 2] & 0xffff0000u);
-                pk[c / 2] = pack_bf16(p0 * (pr[c] - st[c]), p1 * (pr[c + 1] - st[c + 1]));
+                float s0, s1;
+                unpack2(mul2(pack2(p0, p1), fma2(pack2(st[c], st[c + 1]), minus1, pack2(pr[c], pr[c + 1]))), s0, s1);   // p (dP - D)
+                pk[c / 2] = pack_bf16(s0, s1);
             }
             tmem_st32(dp_addr, pk);
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(&bar.ds_full);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar.ds_full);
         }
         // ------------------------------------------------------------ epilogue: warpgroup 0 writes dK, 1 writes dV
         if (ok && E > 0) {
