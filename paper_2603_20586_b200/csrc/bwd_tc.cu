@@ -79,8 +79,8 @@ struct BwdBarriers {
     uint64_t b_full[kMaxStages], b_empty[kMaxStages];     // second streamed ring (dQ kernel: V tiles)
     uint64_t s_full[2];                                   // S landed in TMEM (dQ kernel: ping, pong)
     uint64_t dp_full;                                     // dP landed in TMEM
-    uint64_t p_full;                                      // phase 1 done (dK/dV kernel: P^T written)
-    uint64_t ds_full;                                     // phase 2 done: dS written
+    uint64_t p_part[2];                                   // phase 1 (dK/dV kernel): the first / second 32 columns of every thread's P^T are written
+    uint64_t ds_part[2];                                  // phase 2: the same for dS
     uint64_t acc_done;
 };
 
@@ -212,7 +212,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
             mbar_init(&bar.b_full[s], 1); mbar_init(&bar.b_empty[s], 1);
         }
         mbar_init(&bar.s_full[0], 1); mbar_init(&bar.s_full[1], 1);
-        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 8); mbar_init(&bar.ds_full, 8);   // 8 = one arrival per element-wise warp
+        mbar_init(&bar.dp_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&bar.p_part[i], 8); mbar_init(&bar.ds_part[i], 8); }   // 8 = one arrival per element-wise warp
         mbar_init(&bar.acc_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -301,12 +302,20 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 mma_commit_elect(&bar.dp_full);
                 mma_commit_elect(&bar.b_empty[sv]);
                 if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
-                if (!mbar_wait_warp(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
-                tc_fence_after();
+                // dQ += dS(e) K(e), in the two parts in which the element-wise threads hand dS over (32 of each thread's
+                // 64 columns: K-steps {0, 1, 4, 5}, then {2, 3, 6, 7}), so that the first half runs under the second
 #pragma unroll
-                for (int k = 0; k < kBlk / 16; ++k)         // dQ += dS(e) K(e)
-                    mma_ts_elect(tmem + kColAcc, tmem + kColDP + packed_half_col(k), make_desc(kta + k * (2048 >> 4)), C::kIdescAcc,
-                           (e > 0 || k > 0) ? 1u : 0u);
+                for (int part = 0; part < 2; ++part) {
+                    if (!mbar_wait_warp(&bar.ds_part[part], (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = (i >> 1) * 4 + part * 2 + (i & 1);
+                        mma_ts_elect(tmem + kColAcc, tmem + kColDP + packed_half_col(k), make_desc(kta + k * (2048 >> 4)), C::kIdescAcc,
+                               (e > 0 || part > 0 || i > 0) ? 1u : 0u);
+                    }
+                }
+                if (!ok) break;
                 mma_commit_elect(&bar.a_empty[s]);
             }
             if (ok) mma_commit_elect(&bar.acc_done);
@@ -386,20 +395,30 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dq_tc_kernel(const __grid_con
                 tmem_ld32(dp_addr, reinterpret_cast<uint32_t*>(dp));
                 tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(dp) + 32);
                 tmem_ld_wait();
-                uint32_t pk[32];
+                uint32_t pk[16];
+                auto ds_cols = [&](int c_from, int c_to, int c_base) {
 #pragma unroll
-                for (int c = 0; c < 64; c += 2) {
-                    const uint64_t p2 = pack2(pr[c], pr[c + 1]), d2 = pack2(dp[c], dp[c + 1]);
-                    a2 = fma2(p2, d2, a2);
-                    float s0, s1;
-                    unpack2(mul2(p2, add2(d2, negD2)), s0, s1);
-                    pk[c / 2] = pack_bf16(s0, s1);
-                }
-                tmem_st32(dp_addr, pk);
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bar.ds_full);
+                    for (int c = c_from; c < c_to; c += 2) {
+                        const uint64_t p2 = pack2(pr[c], pr[c + 1]), d2 = pack2(dp[c], dp[c + 1]);
+                        a2 = fma2(p2, d2, a2);
+                        float s0, s1;
+                        unpack2(mul2(p2, add2(d2, negD2)), s0, s1);
+                        pk[(c - c_base) / 2] = pack_bf16(s0, s1);
+                    }
+                };
+                auto hand_over = [&](int part) {
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bar.ds_part[part]);
+                };
+                ds_cols(0, 32, 0);
+                tmem_st16(dp_addr, pk);
+                ds_cols(32, 48, 32);
+                hand_over(0);                                // the first part's store has completed by now
+                ds_cols(48, 64, 32);
+                tmem_st16(dp_addr + 16, pk);
+                hand_over(1);
             }
             {
                 float a0, a1, z0, z1;
@@ -502,7 +521,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
         mbar_init(&bar.fixed_full, 1);
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1); }
         mbar_init(&bar.s_full[0], 1);
-        mbar_init(&bar.dp_full, 1); mbar_init(&bar.p_full, 8); mbar_init(&bar.ds_full, 8);   // 8 = one arrival per element-wise warp
+        mbar_init(&bar.dp_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&bar.p_part[i], 8); mbar_init(&bar.ds_part[i], 8); }   // 8 = one arrival per element-wise warp
         mbar_init(&bar.acc_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -580,19 +600,33 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             for (int e = 0; e < E && ok; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t qta = qt_lo + s * (C::kTile >> 4), gta = gt_lo + s * (C::kTile >> 4);
-                if (!mbar_wait_warp(&bar.p_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
-                tc_fence_after();
+                // dV += P^T(e) dO(e) and dK += dS^T(e) Q(e), each in the two parts in which the element-wise threads
+                // hand their 64 columns over (K-steps {0, 1, 4, 5}, then {2, 3, 6, 7})
 #pragma unroll
-                for (int k = 0; k < kBlk / 16; ++k)         // dV += P^T(e) dO(e)
-                    mma_ts_elect(tmem + kColDV, tmem + kColS + packed_half_col(k), make_desc(gta + k * (2048 >> 4)), C::kIdescAcc,
-                           (e > 0 || k > 0) ? 1u : 0u);
+                for (int part = 0; part < 2; ++part) {
+                    if (!mbar_wait_warp(&bar.p_part[part], (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = (i >> 1) * 4 + part * 2 + (i & 1);
+                        mma_ts_elect(tmem + kColDV, tmem + kColS + packed_half_col(k), make_desc(gta + k * (2048 >> 4)), C::kIdescAcc,
+                               (e > 0 || part > 0 || i > 0) ? 1u : 0u);
+                    }
+                }
+                if (!ok) break;
                 if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
-                if (!mbar_wait_warp(&bar.ds_full, (uint32_t)e & 1u, abortp)) { ok = false; break; }
-                tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < kBlk / 16; ++k)         // dK += dS^T(e) Q(e)
-                    mma_ts_elect(tmem + kColDK, tmem + kColDP + packed_half_col(k), make_desc(qta + k * (2048 >> 4)), C::kIdescAcc,
-                           (e > 0 || k > 0) ? 1u : 0u);
+                for (int part = 0; part < 2; ++part) {
+                    if (!mbar_wait_warp(&bar.ds_part[part], (uint32_t)e & 1u, abortp)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = (i >> 1) * 4 + part * 2 + (i & 1);
+                        mma_ts_elect(tmem + kColDK, tmem + kColDP + packed_half_col(k), make_desc(qta + k * (2048 >> 4)), C::kIdescAcc,
+                               (e > 0 || part > 0 || i > 0) ? 1u : 0u);
+                    }
+                }
+                if (!ok) break;
                 mma_commit_elect(&bar.a_empty[s]);
                 if (e + 1 < E) issue_dp(e + 1);
             }
@@ -657,23 +691,35 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             }
             uint32_t pk[32];        // P^T rounded to bf16; phase 2 uses these same rounded values
             const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
+            auto p_cols = [&](int c_from, int c_to) {
 #pragma unroll
-            for (int c = 0; c < 64; c += 2) {
-                float x0, x1;
-                unpack2(fma2(pack2(pr[c], pr[c + 1]), scale2, pack2(st[c], st[c + 1])), x0, x1);
-                pk[c / 2] = pack_bf16(ex2(x0), ex2(x1));
-            }
-            tmem_st32(s_addr, pk);
+                for (int c = c_from; c < c_to; c += 2) {
+                    float x0, x1;
+                    unpack2(fma2(pack2(pr[c], pr[c + 1]), scale2, pack2(st[c], st[c + 1])), x0, x1);
+                    pk[c / 2] = pack_bf16(ex2(x0), ex2(x1));
+                }
+            };
+            auto hand_over = [&](uint64_t* bar_part) {       // everything stored so far is in TMEM
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_part);
+            };
+            // each half of the thread's 64 columns goes out as soon as it is ready; the first half is handed over in
+            // the middle of the second half's exponentials, when its store has long completed
+            p_cols(0, 32);
+            tmem_st16(s_addr, pk);
+            p_cols(32, 48);
+            hand_over(&bar.p_part[0]);
+            p_cols(48, 64);
+            tmem_st16(s_addr + 16, pk + 16);
             // D_t of the 64 queries, again ahead of the wait
 #pragma unroll
             for (int c = 0; c < 64; c += 4) {
                 const float4 v4 = statD4[c / 4];
                 st[c] = v4.x; st[c + 1] = v4.y; st[c + 2] = v4.z; st[c + 3] = v4.w;
             }
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar.p_full);
+            hand_over(&bar.p_part[1]);
             // phase 2: dS^T = P^T (dP^T - D_t), written over the dP^T columns just read
             ok = mbar_wait(&bar.dp_full, (uint32_t)e & 1u, abortp);
             ok = __all_sync(0xffffffffu, ok);
@@ -683,18 +729,22 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(pr) + 32);
             tmem_ld_wait();
             const uint64_t minus1 = pack2(-1.f, -1.f);
+            auto ds_cols = [&](int c_from, int c_to) {
 #pragma unroll
-            for (int c = 0; c < 64; c += 2) {
-                const float p0 = __uint_as_float(pk[c / 2] << 16), p1 = __uint_as_float(pk[c / 2] & 0xffff0000u);
-                float s0, s1;
-                unpack2(mul2(pack2(p0, p1), fma2(pack2(st[c], st[c + 1]), minus1, pack2(pr[c], pr[c + 1]))), s0, s1);   // p (dP - D)
-                pk[c / 2] = pack_bf16(s0, s1);
-            }
-            tmem_st32(dp_addr, pk);
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar.ds_full);
+                for (int c = c_from; c < c_to; c += 2) {
+                    const float p0 = __uint_as_float(pk[c / 2] << 16), p1 = __uint_as_float(pk[c / 2] & 0xffff0000u);
+                    float s0, s1;
+                    unpack2(mul2(pack2(p0, p1), fma2(pack2(st[c], st[c + 1]), minus1, pack2(pr[c], pr[c + 1]))), s0, s1);   // p (dP - D)
+                    pk[c / 2] = pack_bf16(s0, s1);
+                }
+            };
+            ds_cols(0, 32);
+            tmem_st16(dp_addr, pk);
+            ds_cols(32, 48);
+            hand_over(&bar.ds_part[0]);
+            ds_cols(48, 64);
+            tmem_st16(dp_addr + 16, pk + 16);
+            hand_over(&bar.ds_part[1]);
         }
         // ------------------------------------------------------------ epilogue: warpgroup 0 writes dK, 1 writes dV
         if (ok && E > 0) {

@@ -7,21 +7,22 @@
 //     p = 2^(s * tau * log2(e) + log2(lambda_l) - m)  =  lambda_l * exp(s*tau - m')
 // which is exactly the gated, un-normalised weight of Eq. 5.  One normalisation at the end.
 //
-// Warp roles (d = 128: 640 threads, d = 64: 384 threads):
-//   8 warps per query tile   softmax: warp = (query tile, column half, lane quarter); a thread owns 64 key columns of
-//                    one query row (TMEM lane = row).  Reads S from TMEM, applies bias and masks, agrees with the
-//                    row's other thread on the maximum (shared memory + a 256-thread barrier), exp2, packs the
-//                    weights to bf16 and writes them to TMEM in two parts of 32 keys (at d = 128 over the columns S
-//                    occupied), rescales the O accumulator when the running maximum grows by more than 2^8 (lazy
-//                    rescale), and does the epilogue for its half of the row.
+// Warp roles (d = 128: 320 threads, d = 64: 384 threads):
+//   softmax warps    thread = one query row (TMEM lane) x 128 key columns at d = 128 (four warps per query tile), x 64
+//                    columns at d = 64 (eight warps: warp = (column half, lane quarter); the two threads of a row agree
+//                    on the row maximum through shared memory and a 256-thread barrier).  Reads S from TMEM, applies
+//                    bias and masks, running max, exp2, packs the weights to bf16 and writes them to TMEM in parts of
+//                    32 keys (at d = 128 over the columns S occupied), rescales the O accumulator when the running
+//                    maximum grows by more than 2^8 (lazy rescale), and does the epilogue.
 //   next warp        producer: one lane issues the TMA loads of Q and of the K / V tile list into 128-byte-swizzled
 //                    shared-memory rings (one mbarrier pair per stage); with paged levels the whole warp produces.
 //   next warp        issues every tcgen05.mma (the warp runs its loop converged, one elected lane issues):
 //                    S_q = Q_q K^T (both operands from shared memory) and O_q += P_q V (P from TMEM, V from shared
-//                    memory, N-major) in two halves that follow the two parts of P, so that the first half runs under
-//                    the remaining exponentials.  At d = 128 the order is  S0(e)  O1(e-1)  S1(e)  O0(e):  each tile's
+//                    memory, N-major) in pieces that follow the parts of P, so that most of the product runs under the
+//                    remaining exponentials.  At d = 128 the order is  S0(e)  O1(e-1)  S1(e)  O0(e):  each tile's
 //                    softmax overlaps the other tile's products.
-//   two idle warps   complete the last warpgroup, so that registers can be moved between warpgroups (setmaxnreg).
+//   d = 64 only      two idle warps complete the last warpgroup, so that registers can be moved from it to the softmax
+//                    warpgroups (setmaxnreg): two CTAs per SM leave 80 registers per thread at launch.
 // TMEM: S tiles first (128 columns each), then the O accumulators (d columns each); at d = 64 a P region of 64 columns
 // per query tile follows, and S_q(e+1) is multiplied while the softmax of S_q(e) runs (the hand-off is "S is in
 // registers", not "P has been consumed").  d = 128 uses all 512 columns, d = 64 256.
@@ -35,7 +36,6 @@
 namespace mka {
 namespace {
 
-constexpr int kHalfN = kTileN / 2;                   // key columns of one softmax thread
 constexpr uint32_t kPanelBytes = 128 * 128;          // [128 rows][64 bf16] with 128-byte rows
 constexpr float kRescaleThreshold = 8.0f;            // log2 units
 
@@ -67,22 +67,29 @@ struct TcParams {
 
 template <int DH>
 struct Cfg {
-    // d = 128: one CTA per SM with two query tiles (all 512 TMEM columns).  d = 64: the scores of one key tile cost the
-    // special-function unit as much as at d = 128 but only half the tensor work, and the tile lists of the training
-    // shapes are short; there a CTA takes ONE query tile (256 TMEM columns) and two CTAs share the SM, so that one CTA's
-    // start-up, waits and epilogue run under the other's steady state.
+    // d = 128: one CTA per SM with two query tiles (all 512 TMEM columns); a softmax thread owns a whole query row
+    // (128 key columns, 168 registers per thread).
+    // d = 64: the scores of one key tile cost the special-function unit as much as at d = 128 but only half the
+    // tensor work, and the tile lists of the training shapes are short; there a CTA takes ONE query tile (256 TMEM
+    // columns) and two CTAs share the SM, so that one CTA's start-up, waits and epilogue run under the other's steady
+    // state.  Two CTAs leave 80 registers per thread, so a row is split between two threads (64 columns each), and
+    // registers are moved from the last warpgroup to the softmax warpgroups.
     static constexpr int kNumQ = DH == 128 ? 2 : 1;
     static constexpr int kCtasPerSm = DH == 128 ? 1 : 2;
-    static constexpr int kSoftmaxWarps = 8 * kNumQ;         // per query tile: two column halves x four lane quarters
-    static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;   // one more warpgroup: the producer, the issuing warp, two idle warps
+    static constexpr int kSplit = DH == 128 ? 1 : 2;           // threads per query row
+    static constexpr int kCols = kTileN / kSplit;             // key columns of one softmax thread
+    static constexpr int kParts = kCols / 32;                 // the weights of a tile are handed over in parts of 32 keys per thread
+    static constexpr int kRowWarps = 4 * kSplit;              // softmax warps per query tile
+    static constexpr int kSoftmaxWarps = kRowWarps * kNumQ;
+    static constexpr bool kMoveRegs = kSplit == 2;            // re-divide the registers between the warpgroups (setmaxnreg)
+    // with kMoveRegs the last warpgroup is completed by two idle warps: setmaxnreg is a warpgroup-wide instruction
+    static constexpr int kThreads = (kSoftmaxWarps + (kMoveRegs ? 4 : 2)) * 32;
     static constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
-    // Registers are re-divided between the warpgroups at the start of the kernel: the softmax threads keep 64 scores
-    // and their weights in registers, the last warpgroup needs few.  What the warpgroups hold afterwards must not exceed
-    // what the launch gave the CTA, or the increase would wait forever:
-    //   d = 128: 640 threads x 96 at launch = 512 x 104 + 128 x 64;   d = 64: 384 x 80 = 256 x 104 + 128 x 32.
-    static constexpr int kRegsLaunch = DH == 128 ? 96 : 80, kRegsSoftmax = 104, kRegsOther = DH == 128 ? 64 : 32;
-    static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kThreads * kRegsLaunch, "register pool of the CTA exceeded");
-    static_assert(kThreads * kCtasPerSm * (kRegsLaunch + 8) > 65536, "the launch would get more than kRegsLaunch registers per thread");
+    // What the warpgroups hold after the move must not exceed what the launch gave the CTA, or the increase would
+    // wait forever:  384 threads x 80 registers at launch = 256 x 104 + 128 x 32.
+    static constexpr int kRegsLaunch = 80, kRegsSoftmax = 104, kRegsOther = 32;
+    static_assert(!kMoveRegs || kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kThreads * kRegsLaunch, "register pool of the CTA exceeded");
+    static_assert(!kMoveRegs || kThreads * kCtasPerSm * (kRegsLaunch + 8) > 65536, "the launch would get more than kRegsLaunch registers per thread");
     static constexpr int kPanels = DH / 64;
     static constexpr uint32_t kTileBytes = kPanels * kPanelBytes;
     static constexpr int kStages = 2;
@@ -103,7 +110,7 @@ constexpr int kMaxQ = 2;
 struct Barriers {
     uint64_t q_full;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[kMaxQ], p_part[kMaxQ][2], pv_done[kMaxQ];   // p_part: the first / second 32 keys of both column halves are written
+    uint64_t s_full[kMaxQ], p_part[kMaxQ][4], pv_done[kMaxQ];   // p_part: the first / second 32 keys of both column halves are written
     uint64_t s_free[kMaxQ];   // d = 64 only: the warpgroup has read S(e) into registers, S(e+1) may overwrite it
 };
 
@@ -130,8 +137,8 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
     __shared__ Barriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ WaitCtl wait_ctl;
-    __shared__ float xmax[2][C::kNumQ][2][kTileM];           // row maxima of the two column halves, double-buffered by tile parity
-    __shared__ float lsum[C::kNumQ][2][kTileM];              // row sums of the two column halves (epilogue)
+    __shared__ float xmax[2][C::kNumQ][C::kSplit][kTileM];           // row maxima of the two column halves, double-buffered by tile parity
+    __shared__ float lsum[C::kNumQ][C::kSplit][kTileM];              // row sums of the two column halves (epilogue)
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
@@ -150,8 +157,8 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
         }
         for (int q = 0; q < C::kNumQ; ++q) {
             mbar_init(&bar.s_full[q], 1); mbar_init(&bar.pv_done[q], 1);
-            mbar_init(&bar.p_part[q][0], 8); mbar_init(&bar.p_part[q][1], 8);   // 8 = one arrival per softmax warp
-            mbar_init(&bar.s_free[q], 8);
+            for (int i = 0; i < 4; ++i) mbar_init(&bar.p_part[q][i], C::kRowWarps);   // one arrival per softmax warp
+            mbar_init(&bar.s_free[q], C::kRowWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -185,7 +192,7 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
     const int E = (end[0] - first[0]) + (end[1] - first[1]) + (end[2] - first[2]);
 
     if (warp >= C::kSoftmaxWarps) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
+    if constexpr (C::kMoveRegs) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
     if (warp == C::kProducerWarp && kPaged) {
         // Paged levels: the whole warp produces.  Lane i owns box i of every key tile (a box = the rows of one page
         // that fall into the tile): it looks its page up while the warp waits for the stage to drain and issues its
@@ -337,19 +344,18 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
                 }
                 }
             };
-            // O_q += P_q V in two parts: the softmax warps hand over the weights of keys {0-31, 64-95} of the tile (K-steps
-            // 0, 1, 4, 5) before they have finished those of keys {32-63, 96-127} (K-steps 2, 3, 6, 7), so the first half
-            // of the product runs under the remaining exponentials.
+            // O_q += P_q V in parts: the softmax warps hand over the weights of 32 keys per thread at a time (K-steps
+            // 2 part, 2 part + 1 of every thread's columns), so that the product runs under the remaining exponentials.
             auto issue_pv = [&](int q, int s, int e, bool accumulate) -> bool {
                 const uint32_t va = v_lo + s * (C::kTileBytes >> 4);
                 const uint32_t pa = tmem + (C::kSeparateP ? C::kColP + q * (kTileN / 2) : q * kTileN);
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
+                for (int part = 0; part < C::kParts; ++part) {
                     if (!mbar_wait_warp(&bar.p_part[q][part], (uint32_t)e & 1u, abortp)) return false;
                     tc_fence_after();
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int k = (i >> 1) * 4 + part * 2 + (i & 1);
+                    for (int i = 0; i < 2 * C::kSplit; ++i) {
+                        const int k = (i >> 1) * (8 / C::kSplit) + part * 2 + (i & 1);
                         mma_ts_elect(tmem + C::kColO + q * DH, pa + k * 8, make_desc(va + k * (2048 >> 4)), C::kIdescPV,
                                      (accumulate || part > 0 || i > 0) ? 1u : 0u);
                     }
@@ -417,30 +423,31 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
         }
     }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
+        if constexpr (C::kMoveRegs) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
         // ------------------------------------------------------------ softmax warps
-        // Eight warps per query tile: warp = (query tile, column half, lane quarter).  A thread owns 64 key columns of
-        // one query row; the two threads of a row agree on the row maximum through shared memory at a 256-thread
-        // barrier that also carries their "no wait has run out" flags, so that the 256 threads always leave together.
-        const int q = warp >> 3, half = (warp >> 2) & 1;
+        // warp = (query tile, column part, lane quarter); thread = one query row (TMEM lane) x kCols key columns.
+        // With two threads per row (d = 64) they agree on the row maximum through shared memory at a 256-thread barrier
+        // that also carries their "no wait has run out" flags, so that the 256 threads always leave together.
+        const int q = warp / C::kRowWarps, half = (warp >> 2) % C::kSplit;
         const int row_in_tile = (warp & 3) * 32 + lane;
         const int t = (int)m0 + q * kTileM + row_in_tile;    // T < 2^31
         const bool row_valid = t < p.T;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t s_addr = tmem + lane_base + q * kTileN + half * kHalfN;
-        const uint32_t o_addr = tmem + lane_base + C::kColO + q * DH + half * (DH / 2);
-        // where this thread's 64 weights go as 32 bf16 pairs
-        const uint32_t p_addr = (C::kSeparateP ? tmem + lane_base + C::kColP + q * (kTileN / 2) : tmem + lane_base + q * kTileN) + half * (kHalfN / 2);
+        const uint32_t s_addr = tmem + lane_base + q * kTileN + half * C::kCols;
+        const uint32_t o_addr = tmem + lane_base + C::kColO + q * DH + half * (DH / C::kSplit);
+        // where this thread's weights go as bf16 pairs
+        const uint32_t p_addr = (C::kSeparateP ? tmem + lane_base + C::kColP + q * (kTileN / 2) : tmem + lane_base + q * kTileN) + half * (C::kCols / 2);
         const long long tq0 = m0 + (long long)q * kTileM;                      // first row of this query tile
         const long long tq1 = (tq0 + kTileM - 1 < p.T - 1) ? tq0 + kTileM - 1 : p.T - 1;
-        auto pair_all = [&](bool flag) -> bool {                                // AND over the 256 threads of the query tile
+        auto row_all = [&](bool flag) -> bool {                                 // AND over the threads of the query tile
+            if constexpr (C::kSplit == 1) return flag;
             uint32_t out;
             asm volatile("{\n.reg .pred pi, po;\nsetp.ne.u32 pi, %1, 0;\nbar.red.and.pred po, %2, 256, pi;\nselp.u32 %0, 1, 0, po;\n}"
                          : "=r"(out) : "r"((uint32_t)flag), "r"(1 + q) : "memory");
             return out != 0;
         };
 
-        float m_run = -INFINITY, l_run = 0.f;                                    // l_run: this thread's 64 columns only
+        float m_run = -INFINITY, l_run = 0.f;                                    // l_run: this thread's columns only
         bool ok = true, all_ok = true;                                           // ok is warp-uniform
         int e = 0;
         for (int l = 0; l < 3 && all_ok; ++l) {
@@ -466,12 +473,12 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
             }
             for (int kt = first[l]; kt < end[l]; ++kt, ++e) {
                 if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bar.s_full[q], (uint32_t)e & 1u, abortp));
-                float s[kHalfN];
+                float s[C::kCols];
                 float mx = -INFINITY;
                 if (ok) {
                     tc_fence_after();
 #pragma unroll
-                    for (int c0 = 0; c0 < kHalfN; c0 += 32) tmem_ld32(s_addr + c0, reinterpret_cast<uint32_t*>(s) + c0);
+                    for (int c0 = 0; c0 < C::kCols; c0 += 32) tmem_ld32(s_addr + c0, reinterpret_cast<uint32_t*>(s) + c0);
                     tmem_ld_wait();
                     if (C::kSeparateP) {                     // S(e) is in registers: its TMEM columns may be reused
                         tc_fence_before();
@@ -480,27 +487,30 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
                     }
                     const bool need_mask = !(kt >= full_first && kt < full_end);
                     if (need_mask) {
-                        const long long col0 = (long long)kt * kTileN + half * kHalfN;
-                        const int c_lo = (int)max(-1LL, min((long long)lo - col0, (long long)kHalfN));
-                        const int c_hi = (int)max(-1LL, min((long long)hi - col0, (long long)kHalfN));
+                        const long long col0 = (long long)kt * kTileN + half * C::kCols;
+                        const int c_lo = (int)max(-1LL, min((long long)lo - col0, (long long)C::kCols));
+                        const int c_hi = (int)max(-1LL, min((long long)hi - col0, (long long)C::kCols));
 #pragma unroll
-                        for (int c = 0; c < kHalfN; ++c)
+                        for (int c = 0; c < C::kCols; ++c)
                             if (c < c_lo || c >= c_hi) s[c] = -INFINITY;
                     }
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int c = 0; c < kHalfN; c += 8) {
+                    for (int c = 0; c < C::kCols; c += 8) {
                         mx4[0] = max3(mx4[0], s[c], s[c + 1]); mx4[1] = max3(mx4[1], s[c + 2], s[c + 3]);
                         mx4[2] = max3(mx4[2], s[c + 4], s[c + 5]); mx4[3] = max3(mx4[3], s[c + 6], s[c + 7]);
                     }
                     mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 }
-                // With P written over S (d = 128) this barrier is also what lets a thread overwrite columns that the
-                // other half of its row has read: both halves have their scores in registers when it completes.
-                xmax[e & 1][q][half][row_in_tile] = mx;
-                all_ok = pair_all(ok);
-                if (!all_ok) break;
-                mx = fmaxf(mx, xmax[e & 1][q][half ^ 1][row_in_tile]);
+                if constexpr (C::kSplit == 2) {
+                    xmax[e & 1][q][half][row_in_tile] = mx;
+                    all_ok = row_all(ok);
+                    if (!all_ok) break;
+                    mx = fmaxf(mx, xmax[e & 1][q][half ^ 1][row_in_tile]);
+                } else {
+                    all_ok = ok;
+                    if (!all_ok) break;
+                }
                 const float x_max = fmaf(mx, p.scale_log2, bias);            // -inf when the whole row is masked
                 const float m_new = fmaxf(m_run, x_max);
                 const bool grow = m_new > m_run + kRescaleThreshold;         // also true for the first finite max
@@ -519,7 +529,7 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
                 if (ok) {
                     if (rescale) {                           // some row of this warp moved its reference maximum
 #pragma unroll 1
-                        for (int c0 = 0; c0 < DH / 2; c0 += 32) {
+                        for (int c0 = 0; c0 < DH / C::kSplit; c0 += 32) {
                             uint32_t o[32];
                             tmem_ld32(o_addr + c0, o);
                             tmem_ld_wait();
@@ -528,9 +538,9 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
                             tmem_st32(o_addr + c0, o);
                         }
                     }
-                    // 64 weights in two parts of 32 (16 packed pairs, one store each).  The first part is handed over
-                    // in the middle of the second part's exponentials, when its store has long completed.
-                    // scale, shift and the row sum work on packed pairs: one instruction for two columns
+                    // The weights leave in parts of 32 columns (16 packed pairs, one store each).  A part is handed to
+                    // the issuing warp in the middle of the next part's exponentials, when its store has long completed.
+                    // Scale, shift and the row sum work on packed pairs: one instruction for two columns.
                     const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), shift2 = pack2(shift, shift);
                     uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
                     uint32_t pk[16];
@@ -547,40 +557,42 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
                             pk[(c - c_base) / 2 + 1] = pack_bf16(p2, p3);
                         }
                     };
-                    weights(0, 32, 0);
-                    tmem_st16(p_addr, pk);
-                    weights(32, 48, 32);
-                    tmem_st_wait();                          // the first part (and a rescaled accumulator) is in TMEM
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bar.p_part[q][0]);
-                    weights(48, 64, 32);
-                    tmem_st16(p_addr + 16, pk);
+                    auto hand_over = [&](int part) {         // the part (and a rescaled accumulator) is in TMEM
+                        tmem_st_wait();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bar.p_part[q][part]);
+                    };
+#pragma unroll
+                    for (int part = 0; part < C::kParts; ++part) {
+                        weights(32 * part, 32 * part + 16, 32 * part);
+                        if (part > 0) hand_over(part - 1);
+                        weights(32 * part + 16, 32 * part + 32, 32 * part);
+                        tmem_st16(p_addr + 16 * part, pk);
+                    }
                     {
                         float a0, a1;
                         unpack2(add2(sum_a, sum_b), a0, a1);
                         l_run += a0 + a1;
                     }
-                    tmem_st_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bar.p_part[q][1]);
+                    hand_over(C::kParts - 1);
                 }
             }
         }
         // ------------------------------------------------------------ epilogue
         if (all_ok) {
             if (ok && E > 0) ok = __all_sync(0xffffffffu, mbar_wait(&bar.pv_done[q], (uint32_t)(E - 1) & 1u, abortp));
-            lsum[q][half][row_in_tile] = l_run;              // the row's sum is the sum of its two halves
-            all_ok = pair_all(ok);
+            if constexpr (C::kSplit == 2) lsum[q][half][row_in_tile] = l_run;   // the row's sum is the sum of its two halves
+            all_ok = row_all(ok);
         }
         if (all_ok) {
             tc_fence_after();
-            const float l_row = l_run + lsum[q][half ^ 1][row_in_tile];
+            float l_row = l_run;
+            if constexpr (C::kSplit == 2) l_row += lsum[q][half ^ 1][row_in_tile];
             const float inv = l_row > 0.f ? 1.f / l_row : 0.f;   // rows with nothing visible: exact zeros
-            __nv_bfloat16* Orow = p.O + (((long long)b * p.H + h) * p.T + t) * DH + half * (DH / 2);
+            __nv_bfloat16* Orow = p.O + (((long long)b * p.H + h) * p.T + t) * DH + half * (DH / C::kSplit);
 #pragma unroll 1
-            for (int c0 = 0; c0 < DH / 2; c0 += 32) {
+            for (int c0 = 0; c0 < DH / C::kSplit; c0 += 32) {
                 uint32_t o[32];
                 if (E > 0) {
                     tmem_ld32(o_addr + c0, o);
