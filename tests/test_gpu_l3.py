@@ -26,6 +26,9 @@ CASES = [
     RecallConfig("t_128", 32, 1, 16, 1, 128, 129, 4, 128, 5),
     RecallConfig("t_256", 33, 2, 4, 4, 64, 70, 32, 256, 64, len_frac=(1.0, 0.9)),   # R = 64 = most of the bank
     RecallConfig("t_g7", 34, 2, 28, 4, 128, 2000, 16, 64, 8),
+    # a 16 KB chunk (64 rows of 128), and 128-bit codes over many batches with a partly used and an empty bank
+    RecallConfig("t_p64", 37, 1, 4, 2, 128, 300, 64, 64, 8),
+    RecallConfig("t_b128", 38, 3, 8, 2, 128, 333, 8, 128, 8, len_frac=(1.0, 0.3, 0.0)),
 ]
 
 
