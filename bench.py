@@ -54,14 +54,15 @@ def load_peaks():
 # after the capture.
 NCU_TRAFFIC = {
     # kernel@workload: (bytes in the capture, units of the capture, summary file under profiles/)
-    "fwd_tc_kernel@c3": (376.360448e6 + 66.204160e6, 1 * 8, "fwd_tc_kernel_c3p.md"),
+    "fwd_tc_kernel@c3": (376.982016e6 + 62.288128e6, 1 * 8, "fwd_tc_kernel_c3p.md"),
     "decode_partial_kernel@c4": (1.476463e9 + 5.216768e6, 2 * 32, "decode_partial_kernel_c4p.md"),
-    "bwd_dq_tc_kernel@c5": (220.282624e6 + 29.623808e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
+    "bwd_dq_tc_kernel@c5": (220.273664e6 + 28.019456e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
     "l2_summary_seg_kernel@s3": (100.972800e6 + 55.965184e6, 12288.0 / 32768.0, "l2_summary_seg_kernel_s3p.md"),   # 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8, "fuse_kv_kernel_f3p.md"),
     "decode_paged_kernel@g4": (293.713664e6 + 3.592192e6, 1 * 4, "decode_paged_kernel_g4p.md"),   # one of the four sequences (g4p)
     "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1, "l3_index_kernel_r3p.md"),            # one of the four sequences (r3p)
-    "bwd_dkv_tc_kernel@c5": (220.432640e6 + 115.097856e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
+    "bwd_dkv_tc_kernel@c5": (220.422912e6 + 117.266944e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
+    "fwd_tc_kernel64@c2": (201.660416e6 + 26.980864e6, 8 * 16, "fwd_tc_kernel64_c2.md"),               # the whole configuration
 }
 
 
@@ -412,7 +413,8 @@ def leg_report(leg, ms_per_step, n_gpus, peaks):
         work = w["fwd_flops"] + (w["bwd_flops"] if leg.kind == "train" else 0.0)
         unit, metric = "TFLOP/s", ("fwd_bwd_tflops" if leg.kind == "train" else "prefill_fwd_tflops")
         roof = _tensor_roof("fwd_tc_kernel", w["fwd_flops"] / (k["main"] * 1e-3) / 1e12, peaks,
-                            ncu_traffic("fwd_tc_kernel@c3", cfg) if tag == "c3" else none)
+                            ncu_traffic("fwd_tc_kernel@c3", cfg) if tag == "c3" else
+                            (ncu_traffic("fwd_tc_kernel64@c2", cfg) if leg.name == "c2" else none))
     scale = 1e9 if unit == "GB/s" else 1e12
     value = n_gpus * work / (ms_per_step * 1e-3) / scale
     st = leg.step_stats()
