@@ -59,7 +59,7 @@ NCU_TRAFFIC = {
     "bwd_dq_tc_kernel@c5": (220.273664e6 + 28.019456e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
     "l2_summary_seg_kernel@s3": (100.972800e6 + 55.965184e6, 12288.0 / 32768.0, "l2_summary_seg_kernel_s3p.md"),   # 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8, "fuse_kv_kernel_f3p.md"),
-    "decode_paged_kernel@g4": (293.713664e6 + 3.592192e6, 1 * 4, "decode_paged_kernel_g4p.md"),   # one of the four sequences (g4p)
+    "decode_paged_kernel@g4": (293.682688e6 + 3.988480e6, 1 * 4, "decode_paged_kernel_g4p.md"),   # one of the four sequences (g4p)
     "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1, "l3_index_kernel_r3p.md"),            # one of the four sequences (r3p)
     "bwd_dkv_tc_kernel@c5": (220.422912e6 + 117.266944e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
     "fwd_tc_kernel64@c2": (201.660416e6 + 26.980864e6, 8 * 16, "fwd_tc_kernel64_c2.md"),               # the whole configuration
@@ -395,7 +395,7 @@ def leg_report(leg, ms_per_step, n_gpus, peaks):
                          ncu_traffic("l3_index_kernel@r3", cfg) if tag == "r3" else none)
     elif leg.kind == "paged":
         work, unit, metric = w["decode_bytes"], "GB/s", "decode_paged_hbm_gbs"
-        roof = _hbm_roof("decode_paged_kernel+decode_combine_kernel", work / (k["main"] * 1e-3) / 1e9, peaks,
+        roof = _hbm_roof("decode_paged_tma_kernel+decode_combine_kernel", work / (k["main"] * 1e-3) / 1e9, peaks,
                          ncu_traffic("decode_paged_kernel@g4", cfg) if tag == "g4" else none)
     elif leg.kind == "summary":
         work, unit, metric = w["summary_bytes"], "GB/s", "l2_summary_hbm_gbs"

@@ -248,6 +248,7 @@ mka_status mka_decode(const mka_shape* s, const void* q, const mka_level L[3], c
         pp.q = q; pp.gate = gate; pp.B = s->B; pp.H = s->H; pp.H_kv = s->kv_heads; pp.d = s->d; pp.scale = resolve_scale(s);
         pp.chunk_rows = plan.chunk_rows; pp.total_chunks = plan.total_chunks;
         pp.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeader);
+        pp.status = static_cast<unsigned int*>(ws); pp.wait_limit_ns = wait_limit_ns();
         DecodeParams c;
         memset(&c, 0, sizeof(c));
         c.O = O; c.LSE = LSE; c.gate = gate; c.B = s->B; c.H = s->H; c.d = s->d;

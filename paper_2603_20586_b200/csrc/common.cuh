@@ -125,6 +125,8 @@ struct DecodePagedParams {
     long long n_chunks[3];
     long long total_chunks;
     float* partial;      // [B*H, total_chunks, d+2]
+    unsigned int* status;              // device status word of the call's workspace (bounded waits of the copy-engine form)
+    unsigned long long wait_limit_ns;
 };
 cudaError_t launch_decode_paged(const DecodePagedParams& p, cudaStream_t st);
 cudaError_t launch_l3_index(const void* k, long long n_pages, int H_kv, int page_rows, int d, long long sp, long long sh,

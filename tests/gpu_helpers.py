@@ -46,3 +46,19 @@ def check(gpu, ref, dtype, what=""):
 
 def np64(t):
     return t.detach().double().cpu().numpy()
+
+
+def poison_unused_pool_rows(P, cfg, rows):
+    """NaN into every pool row that no sequence owns: the rows after a sequence's last row inside its last page, and
+    every page that no table entry in use points to (a serving engine's recycled or never-written pages)."""
+    for l in range(3):
+        pk, pv, tab = P["pools_k"][l], P["pools_v"][l], P["tables"][l].cpu().numpy()
+        used = np.zeros((pk.shape[0], cfg.page_rows), dtype=bool)
+        for b in range(cfg.B):
+            n = int(rows[l][b])
+            r = np.arange(n)
+            used[tab[b, r // cfg.page_rows], r % cfg.page_rows] = True
+        dead = torch.from_numpy(~used).to(pk.device)
+        assert bool(dead.any())
+        pk.permute(0, 2, 1, 3)[dead] = float("nan")
+        pv.permute(0, 2, 1, 3)[dead] = float("nan")

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_helpers import check, np64
+from gpu_helpers import check, np64, poison_unused_pool_rows
 from mka_inputs import PAGED_CONFIGS, PagedConfig, make_paged
 
 pytestmark = pytest.mark.gpu
@@ -153,3 +153,24 @@ def test_paged_decode_rejects_bad_arguments(mka):
         mka.mka_decode_paged(shape, 2, P["q"], P["pools_k"], P["pools_v"], P["tables"], list(cfg.N), gate,
                              ws=torch.empty(64, dtype=torch.uint8, device="cuda"))
     assert e.value.code == 4
+
+
+@pytest.mark.parametrize("cfg", [
+    PagedConfig("t_nan16", 23, 2, 8, 2, 128, (300, 2500, 90), 16, rows_frac=(1.0, 0.73)),      # the copy-engine kernel
+    PagedConfig("t_nan256", 24, 2, 6, 2, 64, (700, 3000, 300), 256, rows_frac=(0.9, 1.0)),     # pages longer than a tile
+    PagedConfig("t_nan4", 25, 2, 4, 2, 64, (70, 500, 30), 4, rows_frac=(1.0, 0.6)),            # small pages: the cp.async kernel
+], ids=lambda c: c.name)
+def test_paged_decode_ignores_rows_after_a_sequence_end(mka, orc, cfg):
+    """Pool rows that no sequence owns (the rest of a partly filled last page, unused pages) hold NaN: their weights are
+    zero and they must not reach the output through 0 x NaN in the value product."""
+    P = make_paged(cfg, "cuda")
+    gate = _gate(P)
+    rows = [r.cpu().numpy() for r in P["rows"]]
+    poison_unused_pool_rows(P, cfg, rows)
+    O, LSE = _run(mka, cfg, P, gate)
+    assert bool(torch.isfinite(O.float()).all()) and bool(torch.isfinite(LSE).all())
+    clean = {**P, "pools_k": [torch.nan_to_num(k, nan=0.0) for k in P["pools_k"]],
+             "pools_v": [torch.nan_to_num(v, nan=0.0) for v in P["pools_v"]]}       # the oracle never gathers those rows either
+    Or, Lr = _oracle(orc, cfg, clean, gate)
+    check(O, Or, torch.bfloat16, "paged decode, poisoned tails")
+    assert np.abs(np64(LSE) - Lr).max() <= 2e-3

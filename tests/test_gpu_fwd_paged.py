@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_helpers import check, np64
+from gpu_helpers import check, np64, poison_unused_pool_rows
 from mka_inputs import PagedConfig, approx_normal, make_paged
 
 pytestmark = pytest.mark.gpu
@@ -63,22 +63,6 @@ def test_paged_forward_with_a_length_per_sequence(mka, orc):
     assert np.array_equal(np.isfinite(np64(LSE)), live) and np.abs(np64(LSE)[live] - Lr[live]).max() <= 2e-3
 
 
-def _poison_unused(P, cfg, rows):
-    """NaN into every pool row that no sequence owns: the rows after a sequence's last row inside its last page, and
-    every page that no table entry in use points to (a serving engine's recycled or never-written pages)."""
-    for l in range(3):
-        pk, pv, tab = P["pools_k"][l], P["pools_v"][l], P["tables"][l].cpu().numpy()
-        used = np.zeros((pk.shape[0], cfg.page_rows), dtype=bool)
-        for b in range(cfg.B):
-            n = int(rows[l][b])
-            r = np.arange(n)
-            used[tab[b, r // cfg.page_rows], r % cfg.page_rows] = True
-        dead = torch.from_numpy(~used).to(pk.device)
-        assert bool(dead.any())
-        pk.permute(0, 2, 1, 3)[dead] = float("nan")
-        pv.permute(0, 2, 1, 3)[dead] = float("nan")
-
-
 @pytest.mark.parametrize("cfg,T,W", [
     (PagedConfig("f_nan16", 59, 2, 4, 2, 128, (300, 300, 90), 16, rows_frac=(1.0, 0.7)), 300, 70),
     (PagedConfig("f_nan256", 60, 2, 6, 1, 64, (700, 700, 300), 256, rows_frac=(0.9, 1.0)), 700, 100),
@@ -88,7 +72,7 @@ def test_paged_forward_ignores_rows_after_a_sequence_end(mka, orc, cfg, T, W):
     reach the output through 0 x NaN in the value product."""
     P, Q, gate = _inputs(cfg, T, cfg.seed)
     rows = [r.cpu().numpy() for r in P["rows"]]
-    _poison_unused(P, cfg, rows)
+    poison_unused_pool_rows(P, cfg, rows)
     ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
     O, LSE = mka.mka_fwd_paged(mka.make_shape(cfg.B, cfg.H, T, cfg.d, 32, W), cfg.H_kv, Q, P["pools_k"], P["pools_v"], P["tables"],
                                list(cfg.N), gate, rows=P["rows"], ws=ws)
