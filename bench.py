@@ -50,27 +50,39 @@ def load_peaks():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures summarised under
 # profiles/.  The captures run the profiler-sized workloads (c3p, c4p, c5p, ...: the same per-head geometry with fewer
 # heads / sequences); traffic grows in proportion to the number of units (batch x head pairs, sequences, KV heads), so
-# a full launch is the captured figure times the ratio below.  An entry is dropped (None) when its kernel changes
-# after the capture.
+# a full launch is the captured figure times the ratio below.  Every entry carries a digest of the kernel's source file
+# as it was when the counters were taken: when the file has changed since, the figure is reported as null ("stale").
 NCU_TRAFFIC = {
-    # kernel@workload: (bytes in the capture, units of the capture, summary file under profiles/)
-    "fwd_tc_kernel@c3": (376.982016e6 + 62.288128e6, 1 * 8, "fwd_tc_kernel_c3p.md"),
-    "decode_partial_kernel@c4": (1.476463e9 + 5.216768e6, 2 * 32, "decode_partial_kernel_c4p.md"),
-    "bwd_dq_tc_kernel@c5": (220.273664e6 + 28.019456e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
-    "l2_summary_seg_kernel@s3": (100.972800e6 + 55.965184e6, 12288.0 / 32768.0, "l2_summary_seg_kernel_s3p.md"),   # 12288 of the 32768 tokens
-    "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8, "fuse_kv_kernel_f3p.md"),
-    "decode_paged_kernel@g4": (293.682688e6 + 3.988480e6, 1 * 4, "decode_paged_kernel_g4p.md"),   # one of the four sequences (g4p)
-    "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1, "l3_index_kernel_r3p.md"),            # one of the four sequences (r3p)
-    "bwd_dkv_tc_kernel@c5": (220.422912e6 + 117.266944e6, 1 * 16, "bwd_tc_kernels_c5p.md"),
-    "fwd_tc_kernel64@c2": (201.660416e6 + 26.980864e6, 8 * 16, "fwd_tc_kernel64_c2.md"),               # the whole configuration
+    # kernel@workload: (bytes in the capture, units of the capture, summary file under profiles/, source file, its digest)
+    "fwd_tc_kernel@c3": (376.982016e6 + 62.288128e6, 1 * 8, "fwd_tc_kernel_c3p.md", "fwd_tc.cu", "4df42320d371"),
+    "fwd_tc_kernel64@c2": (201.660416e6 + 26.980864e6, 8 * 16, "fwd_tc_kernel64_c2.md", "fwd_tc.cu", "4df42320d371"),   # the whole configuration
+    "decode_partial_kernel@c4": (1.476476e9 + 5.132288e6, 2 * 32, "decode_partial_kernel_c4p.md", "decode.cu", "ed9d09920f1b"),
+    "bwd_dq_tc_kernel@c5": (220.273664e6 + 28.019456e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "7422e8f986e7"),
+    "bwd_dkv_tc_kernel@c5": (220.422912e6 + 117.266944e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "7422e8f986e7"),
+    "l2_summary_seg_kernel@s3": (101.000704e6 + 55.384064e6, 12288.0 / 32768.0, "l2_summary_seg_kernel_s3p.md", "summary_seg.cu", "6e2dcc00fbde"),   # 12288 of the 32768 tokens
+    "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8, "fuse_kv_kernel_f3p.md", "fuse_kv.cu", "3becacc721a4"),
+    "decode_paged_kernel@g4": (293.682688e6 + 3.988480e6, 1 * 4, "decode_paged_kernel_g4p.md", "decode_paged.cu", "712e1e791061"),   # one of the four sequences (g4p)
+    "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1, "l3_index_kernel_r3p.md", "l3.cu", "614940969b90"),            # one of the four sequences (r3p)
 }
 
 
+def _source_digest(name):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2603_20586_b200", "csrc", name)
+    try:
+        with open(path, "rb") as f:
+            return hashlib.sha256(f.read()).hexdigest()[:12]
+    except OSError:
+        return None
+
+
 def ncu_traffic(key, cfg):
-    """(bytes per full launch, where the figure comes from) or (None, None)."""
+    """(bytes per full launch, where the figure comes from), or (None, why not)."""
     ent = NCU_TRAFFIC.get(key)
     if ent is None:
         return None, None
+    if _source_digest(ent[3]) != ent[4]:
+        return None, f"stale: {ent[3]} has changed since the capture in profiles/{ent[2]}"
     if key.startswith("l3_index"):
         units = cfg.B                                                      # one sequence's bank
     elif key.startswith("decode_paged"):
@@ -429,7 +441,8 @@ def leg_report(leg, ms_per_step, n_gpus, peaks):
         tq, sq = ncu_traffic("bwd_dq_tc_kernel@c5", cfg)
         tkv, _ = ncu_traffic("bwd_dkv_tc_kernel@c5", cfg)
         both = tq is not None and tkv is not None and tag == "c5"
-        rep["roofline_bwd"] = _tensor_roof("bwd_dq_tc_kernel+bwd_dkv_tc_kernel", ach, peaks, ((tq + tkv), sq) if both else none)
+        rep["roofline_bwd"] = _tensor_roof("bwd_dq_tc_kernel+bwd_dkv_tc_kernel", ach, peaks,
+                                           ((tq + tkv), sq) if both else ((None, sq) if tag == "c5" else none))
         rep["roofline_bwd"]["executed_tflops"] = ach * leg.bwd_executed_ratio
     return rep
 
@@ -607,7 +620,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--source-digests", action="store_true", help="print the digests of the kernel sources (for NCU_TRAFFIC) and exit")
     args = ap.parse_args()
+    if args.source_digests:
+        for name in sorted({e[3] for e in NCU_TRAFFIC.values()}):
+            print(name, _source_digest(name))
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

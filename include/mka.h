@@ -195,6 +195,10 @@ typedef struct mka_paged_level {
  *   ws: mka_decode_paged_workspace_bytes(shape, H_kv, n_level) bytes, n_level[l] = L[l].n.  The levels are split into
  *       chunks of a multiple of 128 rows (at most 8192), chosen so that the grid makes few rounds of the resident CTAs
  * d must be 64 or 128; pools 16-byte aligned with strides that are multiples of 8 elements.
+ * Levels whose pages hold at least 8 rows (and dense levels, see mka_decode) are streamed by the copy engine: a
+ * producing warp issues one tensor-map copy per page and 64-column panel, the computing warps wait on barriers for
+ * them.  Those waits are bounded (mka_set_wait_limit_us; mka_device_status(ws) then reads MKA_ERR_TIMEOUT).  Rows of a
+ * partly filled page after a sequence's last row may hold anything, NaN included; pages without a valid row are never read.
  */
 size_t mka_decode_paged_workspace_bytes(const mka_shape* shape, int32_t H_kv, const int64_t n_level[3]);
 mka_status mka_decode_paged(const mka_shape* shape, int32_t H_kv, const void* q, const mka_paged_level L[3],
