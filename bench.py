@@ -333,6 +333,16 @@ class Leg:
             e[3].record()
             self.ev.append(e)
 
+    def rebind(self, t):
+        """Makes `t` (a dict with the same names and shapes) the step's input tensors."""
+        self.t = t
+        if self.kind in ("paged", "recall", "summary"):
+            return
+        self.K = [t["K1"], t["K2"], t["K3"]]
+        self.V = [t["V1"], t["V2"], t["V3"]]
+        if self.kind == "decode":
+            self.q = t["Q"].view(self.cfg.B, self.cfg.H, self.cfg.d)
+
     def result_tensor(self):
         if self.kind in ("paged", "recall"):
             return self.Od
@@ -448,29 +458,53 @@ def leg_report(leg, ms_per_step, n_gpus, peaks):
 
 
 def e2e_run(leg, steps, warmup):
-    """Same step with pinned host inputs: H2D of every input and D2H of the result inside the timed region."""
+    """The same step fed from pinned HOST buffers, through the public binding: every step's inputs are copied host to
+    device and its result device to host inside the timed region.  Two device buffer sets: the copy of step i + 1's
+    inputs (on a second stream) overlaps the kernels of step i, as a serving or training loop would pipeline it.  The
+    timed region starts with an empty pipeline (the first copy overlaps nothing) and ends when the last result is on
+    the host."""
     names = list(leg.t.keys())
     host = {n: torch.empty(leg.t[n].shape, dtype=leg.t[n].dtype, pin_memory=True).copy_(leg.t[n]) for n in names}
+    sets = [leg.t, {n: torch.empty_like(leg.t[n]) for n in names}]
     res = leg.result_tensor()
     host_out = torch.empty(res.shape, dtype=res.dtype, pin_memory=True)
     h2d = sum(h.numel() * h.element_size() for h in host.values())
     d2h = host_out.numel() * host_out.element_size()
+    cur, cp = torch.cuda.current_stream(), torch.cuda.Stream()
+    landed = [torch.cuda.Event() for _ in range(2)]       # the inputs of set k are on the device
+    freed = [torch.cuda.Event() for _ in range(2)]        # the kernels that read set k have finished
 
-    def one():
-        for n in names:
-            leg.t[n].copy_(host[n], non_blocking=True)
+    def upload(k):
+        cp.wait_event(freed[k])
+        with torch.cuda.stream(cp):
+            for n in names:
+                sets[k][n].copy_(host[n], non_blocking=True)
+            landed[k].record(cp)
+
+    def run(k):
+        cur.wait_event(landed[k])
+        leg.rebind(sets[k])
         leg.step()
+        freed[k].record(cur)
         host_out.copy_(leg.result_tensor(), non_blocking=True)
 
-    for _ in range(warmup):
-        one()
+    def loop(n):
+        for k in range(2):
+            freed[k].record(cur)
+        upload(0)
+        for i in range(n):
+            if i + 1 < n:
+                upload((i + 1) & 1)
+            run(i & 1)
+
+    loop(max(2, warmup))
     torch.cuda.synchronize()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
-    for _ in range(steps):
-        one()
+    loop(steps)
     t1.record()
     torch.cuda.synchronize()
+    leg.rebind(sets[0])
     return t0.elapsed_time(t1) / steps, h2d, d2h
 
 
@@ -689,7 +723,7 @@ def main():
         out["bwd_tflops"] = rep["bwd_tflops"]
         out["roofline_bwd"] = rep["roofline_bwd"]
     if not args.no_e2e:
-        e_ms, h2d, d2h = e2e_run(leg, max(2, min(args.steps, 5)), 1)
+        e_ms, h2d, d2h = e2e_run(leg, max(4, min(args.steps, 10)), 2)
         w = leg.work
         if wk == "r3":
             ev = world * w["index_bytes"] / (e_ms * 1e-3) / 1e9
@@ -701,7 +735,8 @@ def main():
             ev = world * w["summary_bytes"] / (e_ms * 1e-3) / 1e9
         else:
             ev = world * (w["fwd_flops"] + (w["bwd_flops"] if wk == "c5" else 0.0)) / (e_ms * 1e-3) / 1e12
-        out["e2e"] = {"value": ev, "unit": rep["unit"], "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        out["e2e"] = {"value": ev, "unit": rep["unit"], "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "pipelined": "two device buffer sets: the host-to-device copy of step i + 1 overlaps the kernels of step i"}
     del leg
     torch.cuda.empty_cache()
     if rank == 0 and not args.no_cpu_baseline and world == 1:
