@@ -63,6 +63,7 @@ struct TcParams {
     long long table_stride[3], table_head_stride[3];
     int page_shift[3], box_rows[3], pool_pages[3];
     const int* rows[3];      // per-sequence rows of a level (clamped to [0, n]), or null
+    int deal;                // (batch, head) pairs per group of blocks dealt by query block (1 = pair by pair)
 };
 
 template <int DH>
@@ -142,8 +143,16 @@ __global__ void __launch_bounds__(Cfg<DH>::kThreads, Cfg<DH>::kCtasPerSm) fwd_tc
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // tid >> 5, but provably warp-uniform for the compiler
-    const int b = blockIdx.z, h = blockIdx.y;
-    const int qpair = gridDim.x - 1 - blockIdx.x;          // heaviest (latest) rows first
+    // Blocks start in the order of their linear index.  Within a group of p.deal (batch, head) pairs the blocks are
+    // dealt by query block, heaviest (latest rows) first for every pair of the group, then the next lighter one: the
+    // launch then ends with the group's lightest blocks instead of the last head's heaviest.
+    const int lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);      // fewer than 2^31 blocks
+    const int per_group = p.deal * (int)gridDim.x;
+    const int grp = lin / per_group, in_grp = lin - grp * per_group;
+    const int pairs_here = min(p.deal, (int)(gridDim.y * gridDim.z) - grp * p.deal);
+    const int hb = grp * p.deal + in_grp % pairs_here;
+    const int b = hb / (int)gridDim.y, h = hb - b * (int)gridDim.y;
+    const int qpair = gridDim.x - 1 - in_grp / pairs_here;
     const long long m0 = (long long)qpair * (C::kNumQ * kTileM);
     const long long m_last = (m0 + C::kNumQ * kTileM - 1 < p.T - 1) ? m0 + C::kNumQ * kTileM - 1 : p.T - 1;
 
@@ -665,6 +674,15 @@ cudaError_t launch_t(const FwdParams& fp, unsigned int* status_word, cudaStream_
     p.status = status_word;
     p.wait_limit_ns = wait_limit_ns();
     p.test_stall = fp.test_stall;
+    {   // as many (batch, head) pairs per group as keep the group's K and V (48 MB at most) in the L2 cache while
+        // its blocks, dealt by query block, re-read them
+        double pair_bytes = 0.0;
+        for (int l = 0; l < 3; ++l) pair_bytes += (double)fp.L[l].n * DH * 4.0;
+        pair_bytes /= fp.kv_group;
+        const double pairs = (double)fp.B * fp.H;
+        const double fit = pair_bytes > 0.0 ? 48.0 * 1024 * 1024 / pair_bytes : pairs;
+        p.deal = fit < 1.0 ? 1 : (fit > pairs ? (int)pairs : (int)fit);
+    }
     auto kern = fp.paged ? fwd_tc_kernel<DH, true> : fwd_tc_kernel<DH, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<DH>::kSmemBytes);
     if (e != cudaSuccess) return e;
@@ -679,6 +697,7 @@ bool fwd_tc_eligible(const FwdParams& p, int dtype) {
     if (dtype != MKA_BF16 || p.mode != MKA_MODE_FAST || p.decode) return false;
     if (p.d != 64 && p.d != 128) return false;
     if (p.H > 65535 || p.B > 65535) return false;
+    if ((double)((p.T + 127) / 128) * p.H * p.B > 2147483647.0) return false;   // the kernel numbers its blocks in an int
     for (int l = 0; l < 3; ++l) {
         const LevelDev& L = p.L[l];
         if (L.n == 0) continue;
