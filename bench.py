@@ -54,8 +54,8 @@ def load_peaks():
 # as it was when the counters were taken: when the file has changed since, the figure is reported as null ("stale").
 NCU_TRAFFIC = {
     # kernel@workload: (bytes in the capture, units of the capture, summary file under profiles/, source file, its digest)
-    "fwd_tc_kernel@c3": (376.982016e6 + 62.288128e6, 1 * 8, "fwd_tc_kernel_c3p.md", "fwd_tc.cu", "4df42320d371"),
-    "fwd_tc_kernel64@c2": (201.660416e6 + 26.980864e6, 8 * 16, "fwd_tc_kernel64_c2.md", "fwd_tc.cu", "4df42320d371"),   # the whole configuration
+    "fwd_tc_kernel@c3": (376.523776e6 + 61.946368e6, 1 * 8, "fwd_tc_kernel_c3p.md", "fwd_tc.cu", "58f08d0c47e4"),
+    "fwd_tc_kernel64@c2": (204.546304e6 + 28.208640e6, 8 * 16, "fwd_tc_kernel64_c2.md", "fwd_tc.cu", "58f08d0c47e4"),   # the whole configuration
     "decode_partial_kernel@c4": (1.476476e9 + 5.132288e6, 2 * 32, "decode_partial_kernel_c4p.md", "decode.cu", "ed9d09920f1b"),
     "bwd_dq_tc_kernel@c5": (220.273664e6 + 28.019456e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "7422e8f986e7"),
     "bwd_dkv_tc_kernel@c5": (220.422912e6 + 117.266944e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "7422e8f986e7"),
