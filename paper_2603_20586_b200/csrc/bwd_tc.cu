@@ -17,12 +17,21 @@
 // Both kernels recompute the scores (7 matrix products per visible tile pair instead of 5) in exchange
 // for needing no atomics and no cross-CTA reduction.
 //
+// In the dK/dV kernel the per-query terms vary along the COLUMNS of the transposed tiles, where a thread would need 64
+// biases and 64 D_t per tile from shared memory (which the tensor pipe saturates).  They enter through the tensor pipe
+// instead: both score products get a ninth K-step whose key-side operand is ones and whose query-side operand holds
+// bias_t / scale (for S^T) or -D_t (for dP^T), each split into three bf16 terms, so S^T + bias / scale and dP^T - D arrive
+// in TMEM ready-made.  The producing warp writes those 4 KB operand slabs (no swizzle) from the statistics of the prep
+// kernel, fetched one tile ahead.  Q tiles and dO tiles travel in rings of their own: dO(e) is free again after dV(e),
+// Q(e) only after dK(e), and Q(e+1) is what the next score product waits for.  Half of the exponentials of that kernel
+// run as a cubic on the FMA pipe (exp2_pair_fma).
+//
 // Warp roles (320 threads): warps 0-7 are the element-wise ("softmax") threads: thread i of either
 // warpgroup owns TMEM lane i & 127 (a query row in the dQ kernel, a key row in the dK/dV kernel);
 // warpgroup 0 takes columns 0-63 of a tile and warpgroup 1 columns 64-127.  Their work on a tile has
 // two phases so that it overlaps the tensor pipe: phase 1 needs only S (p = 2^(s*scale + bias), kept in
 // registers) and runs while dP is still being multiplied; phase 2 reads dP, forms dS = p (dP - D) and
-// writes it (bf16) over the columns of dP it has just read.  Warp 8 lane 0 issues the TMA loads;
+// writes it (bf16) over the columns of dP it has just read.  Warp 8 issues the TMA loads (lane 0);
 // warp 9 issues every tcgen05.mma, running its loop converged with one elected lane issuing.
 // TMEM (512 columns), dQ kernel: S ping [0,128), S pong [128,256), dP/dS [256,384), dQ [384,384+d).
 //                     dK/dV kernel: S^T/P^T [0,128), dP^T/dS^T [128,256), dK [256,256+d), dV [256+d,256+2d).
@@ -59,15 +68,46 @@ struct BwdTcParams {
     unsigned long long wait_limit_ns;
 };
 
+// v as a sum of three bf16 terms (exact to 2^-25 |v|) in the first three of eight bf16 slots of a 16-byte core-matrix row;
+// an infinite v (the bias of a padding row or of a level the gate closes) stays one infinite term.
+__device__ __forceinline__ uint4 split3_bf16(float v) {
+    if (!(fabsf(v) <= 3.0e38f)) return make_uint4(pack_bf16(v, 0.f), 0u, 0u, 0u);
+    const float t0 = __bfloat162float(__float2bfloat16_rn(v));
+    const float r1 = v - t0;
+    const float t1 = __bfloat162float(__float2bfloat16_rn(r1));
+    return make_uint4(pack_bf16(t0, t1), pack_bf16(r1 - t1, 0.f), 0u, 0u);
+}
+
+// 2^x for two arguments x <= 0 on the FMA pipe: x is clamped to -127 and split into n = round(x) and f = x - n in
+// [-1/2, 1/2] by adding and subtracting 1.5 * 2^23 (the sum's low mantissa bits are n); 2^f is a cubic with constant term
+// exactly 1 (coefficients fitted for the smallest maximum relative error, 1.0e-4, a twentieth of the rounding step of
+// the bf16 value it becomes); n is added to the exponent field.  x <= -127 gives exactly 0, as ex2 does for -inf.
+__device__ __forceinline__ void exp2_pair_fma(float x0, float x1, float& p0, float& p1) {
+    const float kMagic = 12582912.f;
+    const uint64_t x = pack2(fmaxf(x0, -127.f), fmaxf(x1, -127.f));
+    const uint64_t t = add2(x, pack2(kMagic, kMagic));
+    const uint64_t n = add2(t, pack2(-kMagic, -kMagic));
+    const uint64_t f = fma2(n, pack2(-1.f, -1.f), x);
+    uint64_t r = fma2(pack2(0.05500893f, 0.05500893f), f, pack2(0.24221095f, 0.24221095f));
+    r = fma2(r, f, pack2(0.69328290f, 0.69328290f));
+    r = fma2(r, f, pack2(1.f, 1.f));
+    float r0, r1, t0, t1;
+    unpack2(r, r0, r1);
+    unpack2(t, t0, t1);
+    p0 = __uint_as_float(__float_as_uint(r0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(r1) + (__float_as_uint(t1) << 23));
+}
+
 template <int DH>
 struct BCfg {
     static constexpr int kPanels = DH / 64;
     static constexpr uint32_t kTile = kPanels * kPanel;       // a 128-row tile
     static constexpr int kStages = DH == 128 ? 2 : 4;         // also keeps the CTA above half of shared memory
-    static constexpr uint32_t kStatBytes = 2 * kBlk * sizeof(float);   // per stage: D and the level's bias of 128 queries
+    // dK/dV kernel: the per-query terms enter the two score products as one more K-step (see kAugBytes below)
+    static constexpr uint32_t kAugBytes = kBlk * 16 * 2;              // a [128 rows][16] bf16 operand slab without swizzle
     static constexpr int kStagesK = DH == 128 ? 3 : 4;        // K ring of the dQ kernel: K(e) stays in use until dQ(e), two tiles after it is first read
     static constexpr uint32_t kSmemDq = 2 * kTile + (kStages + kStagesK) * kTile + 1024;
-    static constexpr uint32_t kSmemDkv = 2 * kTile + kStages * (2 * kTile + kStatBytes) + 1024;
+    static constexpr uint32_t kSmemDkv = 2 * kTile + kStages * (2 * kTile + 2 * kAugBytes) + kAugBytes + 1024;
     // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
     static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlk >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     static constexpr uint32_t kIdescAcc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -75,8 +115,8 @@ struct BCfg {
 
 struct BwdBarriers {
     uint64_t fixed_full;                                  // the CTA's own (non-streamed) tiles
-    uint64_t a_full[kMaxStages], a_empty[kMaxStages];     // streamed ring (dQ kernel: K tiles; dK/dV kernel: Q + dO + stats)
-    uint64_t b_full[kMaxStages], b_empty[kMaxStages];     // second streamed ring (dQ kernel: V tiles)
+    uint64_t a_full[kMaxStages], a_empty[kMaxStages];     // streamed ring (dQ kernel: K tiles; dK/dV kernel: Q tiles + bias slabs)
+    uint64_t b_full[kMaxStages], b_empty[kMaxStages];     // second streamed ring (dQ kernel: V tiles; dK/dV kernel: dO tiles + D slabs)
     uint64_t s_full[2];                                   // S landed in TMEM (dQ kernel: ping, pong)
     uint64_t dp_full;                                     // dP landed in TMEM
     uint64_t p_part[2];                                   // phase 1 (dK/dV kernel): the first / second 32 columns of every thread's P^T are written
@@ -84,10 +124,6 @@ struct BwdBarriers {
     uint64_t acc_done;
 };
 
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
 __device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------ prep
@@ -486,7 +522,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     uint8_t* sV = sK + C::kTile;
     uint8_t* sQ = sV + C::kTile;                          // kStages tiles
     uint8_t* sdO = sQ + C::kStages * C::kTile;            // kStages tiles
-    float* sStat = reinterpret_cast<float*>(sdO + C::kStages * C::kTile);     // kStages x {D[128], bias[128]}
+    // Operand slabs of the extra K-step (16 columns, no swizzle: 8-row x 16-byte core matrices, the two of a row group
+    // 128 bytes apart, row groups 256 bytes apart).  sAugQ: per stage, [query][k] = the query's exponent bias divided by
+    // the score scale, split into three bf16 terms (k = 0..2), then [query][k] = -D_t split the same way; sAugK: ones in
+    // k = 0..2 for every key.  S^T + bias / scale and dP^T - D then come out of the tensor pipe, and the element-wise
+    // threads need no per-column operand at all.
+    uint8_t* sAugQ = sdO + C::kStages * C::kTile;          // kStages x {bias slab, D slab}
+    uint8_t* sAugK = sAugQ + C::kStages * 2 * C::kAugBytes;
     __shared__ BwdBarriers bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ WaitCtl wait_ctl;
@@ -519,7 +561,10 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
         wait_ctl.abort = 0;
         wait_ctl.limit_ns = p.wait_limit_ns;
         mbar_init(&bar.fixed_full, 1);
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bar.a_full[s], 1); mbar_init(&bar.a_empty[s], 1); }
+        for (int s = 0; s < kMaxStages; ++s) {               // full: the copy's bytes and the slab
+            mbar_init(&bar.a_full[s], 2); mbar_init(&bar.a_empty[s], 1);
+            mbar_init(&bar.b_full[s], 2); mbar_init(&bar.b_empty[s], 1);
+        }
         mbar_init(&bar.s_full[0], 1);
         mbar_init(&bar.dp_full, 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&bar.p_part[i], 8); mbar_init(&bar.ds_part[i], 8); }   // 8 = one arrival per element-wise warp
@@ -537,37 +582,79 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     volatile WaitCtl* abortp = &wait_ctl;
 
     if (warp == kProducerWarp) {
-        if (lane == 0 && E > 0) {
-            int issued = 0;
-            mbar_expect_tx(&bar.fixed_full, 2 * C::kTile);
+        if (E > 0) {   // the whole warp runs the loop (converged): lane 0 issues the copies, every lane writes its share of the slabs
+            int issued = 0, issued_b = 0;
+            // zero every slab once (columns 3..15 stay zero), ones for the keys
+            for (int i = lane; i < (int)((C::kStages * 2 + 1) * C::kAugBytes / 16); i += 32)
+                reinterpret_cast<uint4*>(sAugQ)[i] = make_uint4(0u, 0u, 0u, 0u);
+            __syncwarp();
+            for (int r = lane; r < kBlk; r += 32)
+                *reinterpret_cast<uint4*>(sAugK + (r & 7) * 16 + (r >> 3) * 256) = make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u);
+            if (lane == 0) {
+                mbar_expect_tx(&bar.fixed_full, 2 * C::kTile);
 #pragma unroll
-            for (int pn = 0; pn < C::kPanels; ++pn) {
-                tma_load_4d(sK + pn * kPanel, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
-                tma_load_4d(sV + pn * kPanel, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                for (int pn = 0; pn < C::kPanels; ++pn) {
+                    tma_load_4d(sK + pn * kPanel, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                    tma_load_4d(sV + pn * kPanel, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                }
             }
+            const float inv_scale = 1.f / p.scale_log2;
             int hq = h * p.kv_group, eq = 0;                // query head and tile-within-head of stage e
+            // this lane's four queries of a tile: their biases and D_t, fetched one tile ahead of the stage they go into
+            auto fetch = [&](float4& bq, float4& dq) {
+                const long long at = ((long long)b * p.H + hq) * p.Tpad + (long long)(first + eq) * kBlk + 4 * lane;
+                bq = *reinterpret_cast<const float4*>(p.statB[lvl] + at);
+                dq = *reinterpret_cast<const float4*>(p.statD + at);
+            };
+            float4 bq, dq;
+            fetch(bq, dq);
+            // Two rings: a stage's dO tile is free again after dV of its tile, its Q tile only after dK, one product later;
+            // and the next tile's Q is what the issuing warp waits for first.  Each is re-filled as soon as it is free.
             for (int e = 0; e < E; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
-                if (!mbar_wait(&bar.a_empty[s], ph ^ 1u, abortp)) break;
-                const long long bh = (long long)b * p.H + hq;
-                const float* statD = p.statD + bh * p.Tpad;
-                const float* statB = p.statB[lvl] + bh * p.Tpad;
                 const int tt = (first + eq) * kBlk;
-                mbar_expect_tx(&bar.a_full[s], 2 * C::kTile + C::kStatBytes);
+                const float bv[4] = {bq.x, bq.y, bq.z, bq.w}, dv[4] = {dq.x, dq.y, dq.z, dq.w};
+                if (!mbar_wait_warp(&bar.b_empty[s], ph ^ 1u, abortp)) break;
+                if (lane == 0) {
+                    mbar_expect_tx(&bar.b_full[s], C::kTile);
 #pragma unroll
-                for (int pn = 0; pn < C::kPanels; ++pn) {
-                    tma_load_4d(sQ + s * C::kTile + pn * kPanel, &maps.q, pn * 64, tt, hq, b, &bar.a_full[s]);
-                    tma_load_4d(sdO + s * C::kTile + pn * kPanel, &maps.dO, pn * 64, tt, hq, b, &bar.a_full[s]);
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sdO + s * C::kTile + pn * kPanel, &maps.dO, pn * 64, tt, hq, b, &bar.b_full[s]);
                 }
-                bulk_load(sStat + s * 2 * kBlk, statD + tt, kBlk * sizeof(float), &bar.a_full[s]);
-                bulk_load(sStat + s * 2 * kBlk + kBlk, statB + tt, kBlk * sizeof(float), &bar.a_full[s]);
+                ++issued_b;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {                          // -D as three bf16 terms
+                    const int r = 4 * lane + i;
+                    *reinterpret_cast<uint4*>(sAugQ + (s * 2 + 1) * C::kAugBytes + (r & 7) * 16 + (r >> 3) * 256) = split3_bf16(-dv[i]);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar.b_full[s]);
+                if (!mbar_wait_warp(&bar.a_empty[s], ph ^ 1u, abortp)) break;
+                if (lane == 0) {
+                    mbar_expect_tx(&bar.a_full[s], C::kTile);
+#pragma unroll
+                    for (int pn = 0; pn < C::kPanels; ++pn)
+                        tma_load_4d(sQ + s * C::kTile + pn * kPanel, &maps.q, pn * 64, tt, hq, b, &bar.a_full[s]);
+                }
                 ++issued;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {                          // bias / scale as three bf16 terms
+                    const int r = 4 * lane + i;
+                    *reinterpret_cast<uint4*>(sAugQ + (s * 2) * C::kAugBytes + (r & 7) * 16 + (r >> 3) * 256) = split3_bf16(bv[i] * inv_scale);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar.a_full[s]);
                 if (++eq == Eq) { eq = 0; ++hq; }
+                if (e + 1 < E) fetch(bq, dq);
             }
-            mbar_wait(&bar.fixed_full, 0, abortp);
+            mbar_wait_warp(&bar.fixed_full, 0, abortp);
             for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
-                mbar_wait(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+                mbar_wait_warp(&bar.a_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
+            for (int i = issued_b > C::kStages ? issued_b - C::kStages : 0; i < issued_b; ++i)
+                mbar_wait_warp(&bar.b_full[i % C::kStages], (uint32_t)(i / C::kStages) & 1u, abortp);
         }
     } else if (warp == kMmaWarp) {
         if (E > 0) {   // every lane runs the issue loop (converged); elect.sync inside the wrappers picks the issuing lane
@@ -577,6 +664,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             const uint32_t k_lo = desc_lo_kmajor(smem_u32(sK)), v_lo = desc_lo_kmajor(smem_u32(sV));
             const uint32_t q_lo = desc_lo_kmajor(smem_u32(sQ)), g_lo = desc_lo_kmajor(smem_u32(sdO));
             const uint32_t qt_lo = desc_lo_mnmajor(smem_u32(sQ), kPanel), gt_lo = desc_lo_mnmajor(smem_u32(sdO), kPanel);
+            const uint32_t augk_lo = desc_lo_flat(smem_u32(sAugK)), augq_lo = desc_lo_flat(smem_u32(sAugQ));
             auto issue_s = [&](int e) -> bool {             // S^T(e) = K Q(e)^T   (P^T(e-1), which shares the columns, was consumed by dV(e-1) issued before)
                 const int s = e % C::kStages;
                 if (!mbar_wait_warp(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
@@ -585,18 +673,23 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
 #pragma unroll
                 for (int k = 0; k < DH / 16; ++k)
                     mma_ss_elect(tmem + kColS, make_desc(k_lo + kstep_off(k, kPanel)), make_desc(qa + kstep_off(k, kPanel)), C::kIdescS, k > 0);
+                mma_ss_elect(tmem + kColS, make_desc_flat(augk_lo), make_desc_flat(augq_lo + s * (2 * C::kAugBytes >> 4)), C::kIdescS, 1u);   // + bias_t / scale
                 mma_commit_elect(&bar.s_full[0]);
                 return true;
             };
-            auto issue_dp = [&](int e) {                    // dP^T(e) = V dO(e)^T  (its stage was awaited by issue_s(e))
+            auto issue_dp = [&](int e) -> bool {            // dP^T(e) = V dO(e)^T
+                if (!mbar_wait_warp(&bar.b_full[e % C::kStages], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
+                tc_fence_after();
                 const uint32_t ga = g_lo + (e % C::kStages) * (C::kTile >> 4);
 #pragma unroll
                 for (int k = 0; k < DH / 16; ++k)
                     mma_ss_elect(tmem + kColDP, make_desc(v_lo + kstep_off(k, kPanel)), make_desc(ga + kstep_off(k, kPanel)), C::kIdescS, k > 0);
+                mma_ss_elect(tmem + kColDP, make_desc_flat(augk_lo), make_desc_flat(augq_lo + ((e % C::kStages) * 2 + 1) * (C::kAugBytes >> 4)), C::kIdescS, 1u);   // - D_t
                 mma_commit_elect(&bar.dp_full);
+                return true;
             };
             if (ok) ok = issue_s(0);
-            if (ok) issue_dp(0);
+            if (ok) ok = issue_dp(0);
             for (int e = 0; e < E && ok; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t qta = qt_lo + s * (C::kTile >> 4), gta = gt_lo + s * (C::kTile >> 4);
@@ -614,6 +707,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                     }
                 }
                 if (!ok) break;
+                mma_commit_elect(&bar.b_empty[s]);                     // dO(e) has had its last reader
                 if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
@@ -628,7 +722,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                 }
                 if (!ok) break;
                 mma_commit_elect(&bar.a_empty[s]);
-                if (e + 1 < E) issue_dp(e + 1);
+                if (e + 1 < E && !issue_dp(e + 1)) { ok = false; break; }
             }
             if (ok) mma_commit_elect(&bar.acc_done);
         }
@@ -654,21 +748,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             const int s = e % C::kStages;
             const long long tt = (long long)(first + eq) * kBlk;       // first query of the tile
             if (++eq == Eq) eq = 0;
-            // The per-query statistics of the tile sit in this stage's shared memory; fetch this thread's 64 biases
-            // before waiting for S so that the loads' latency (long while the tensor pipe saturates shared
-            // memory) is off the path.  The stage's own barrier has long completed; waiting on it orders the reads.
-            ok = mbar_wait(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const float4* statD4 = reinterpret_cast<const float4*>(sStat + s * 2 * kBlk + w * 64);
-            const float4* statB4 = reinterpret_cast<const float4*>(sStat + s * 2 * kBlk + kBlk + w * 64);
-            float st[64];
-#pragma unroll
-            for (int c = 0; c < 64; c += 4) {
-                const float4 v4 = statB4[c / 4];
-                st[c] = v4.x; st[c + 1] = v4.y; st[c + 2] = v4.z; st[c + 3] = v4.w;
-            }
-            // phase 1: P^T = 2^(s * scale + bias_t) for this thread's 64 query columns
+            // phase 1: P^T = 2^(scale * (s + bias_t / scale)) for this thread's 64 query columns; the sum comes from the tensor pipe
             ok = mbar_wait(&bar.s_full[0], (uint32_t)e & 1u, abortp);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -695,8 +775,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
 #pragma unroll
                 for (int c = c_from; c < c_to; c += 2) {
                     float x0, x1;
-                    unpack2(fma2(pack2(pr[c], pr[c + 1]), scale2, pack2(st[c], st[c + 1])), x0, x1);
-                    pk[c / 2] = pack_bf16(ex2(x0), ex2(x1));
+                    unpack2(mul2(pack2(pr[c], pr[c + 1]), scale2), x0, x1);
+                    // Every other pair on the FMA pipe: the hand-over of P^T, not these threads' total work, is what the
+                    // next score product waits for, and the special-function unit alone is the slower way there.
+                    float p0, p1;
+                    if ((c >> 1) & 1) { p0 = ex2(x0); p1 = ex2(x1); }
+                    else exp2_pair_fma(x0, x1, p0, p1);
+                    pk[c / 2] = pack_bf16(p0, p1);
                 }
             };
             auto hand_over = [&](uint64_t* bar_part) {       // everything stored so far is in TMEM
@@ -713,14 +798,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             hand_over(&bar.p_part[0]);
             p_cols(48, 64);
             tmem_st16(s_addr + 16, pk + 16);
-            // D_t of the 64 queries, again ahead of the wait
-#pragma unroll
-            for (int c = 0; c < 64; c += 4) {
-                const float4 v4 = statD4[c / 4];
-                st[c] = v4.x; st[c + 1] = v4.y; st[c + 2] = v4.z; st[c + 3] = v4.w;
-            }
             hand_over(&bar.p_part[1]);
-            // phase 2: dS^T = P^T (dP^T - D_t), written over the dP^T columns just read
+            // phase 2: dS^T = P^T (dP^T - D_t), written over the columns just read; the difference comes from the tensor pipe
             ok = mbar_wait(&bar.dp_full, (uint32_t)e & 1u, abortp);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -728,13 +807,12 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             tmem_ld32(dp_addr, reinterpret_cast<uint32_t*>(pr));
             tmem_ld32(dp_addr + 32, reinterpret_cast<uint32_t*>(pr) + 32);
             tmem_ld_wait();
-            const uint64_t minus1 = pack2(-1.f, -1.f);
             auto ds_cols = [&](int c_from, int c_to) {
 #pragma unroll
                 for (int c = c_from; c < c_to; c += 2) {
                     const float p0 = __uint_as_float(pk[c / 2] << 16), p1 = __uint_as_float(pk[c / 2] & 0xffff0000u);
                     float s0, s1;
-                    unpack2(mul2(pack2(p0, p1), fma2(pack2(st[c], st[c + 1]), minus1, pack2(pr[c], pr[c + 1]))), s0, s1);   // p (dP - D)
+                    unpack2(mul2(pack2(p0, p1), pack2(pr[c], pr[c + 1])), s0, s1);   // p (dP - D)
                     pk[c / 2] = pack_bf16(s0, s1);
                 }
             };

@@ -87,6 +87,15 @@ __device__ __forceinline__ uint32_t desc_lo_kmajor(uint32_t addr) { return (addr
 __device__ __forceinline__ uint32_t desc_lo_mnmajor(uint32_t addr, uint32_t panel_stride_bytes) {
     return (addr >> 4) | ((panel_stride_bytes >> 4) << 16);
 }
+// Descriptor words of a K-major operand slab WITHOUT swizzle, 16 columns (one K-step) wide: core matrices of 8 rows x 16
+// bytes; the two core matrices of a row group lie 128 bytes apart (leading-dimension field), row groups 256 bytes apart.
+constexpr uint32_t kDescHiFlat = (256u >> 4) | (1u << 14);
+__device__ __forceinline__ uint32_t desc_lo_flat(uint32_t addr) { return (addr >> 4) | ((128u >> 4) << 16); }
+__device__ __forceinline__ uint64_t make_desc_flat(uint32_t lo) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(kDescHiFlat));
+    return d;
+}
 __device__ __forceinline__ uint64_t make_desc(uint32_t lo) {
     uint64_t d;
     asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(kDescHi));
