@@ -557,7 +557,9 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     const int Eq = t_hi > t_lo ? (int)((t_hi + kBlk - 1) / kBlk) - first : 0;    // query tiles of ONE head that see this key tile
     const int E = Eq * p.kv_group;                          // the stream: head by head, each head's tiles in order
 
-    if (tid == 0) {
+    // The thread that issues the copies sets the barriers up itself and requests the CTA's own K and V tiles at once,
+    // before the CTA-wide start-up (slabs, TMEM allocation) that the copies' latency can run under.
+    if (warp == kProducerWarp && lane == 0) {
         wait_ctl.abort = 0;
         wait_ctl.limit_ns = p.wait_limit_ns;
         mbar_init(&bar.fixed_full, 1);
@@ -570,7 +572,21 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
         for (int i = 0; i < 2; ++i) { mbar_init(&bar.p_part[i], 8); mbar_init(&bar.ds_part[i], 8); }   // 8 = one arrival per element-wise warp
         mbar_init(&bar.acc_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (E > 0) {
+            mbar_expect_tx(&bar.fixed_full, 2 * C::kTile);
+#pragma unroll
+            for (int pn = 0; pn < C::kPanels; ++pn) {
+                tma_load_4d(sK + pn * kPanel, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+                tma_load_4d(sV + pn * kPanel, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
+            }
+        }
     }
+    // every slab zero (columns 3..15 stay zero), ones for the keys: all threads share the 36 KB
+    for (int i = tid; i < (int)((C::kStages * 2 + 1) * C::kAugBytes / 16); i += kThreads)
+        reinterpret_cast<uint4*>(sAugQ)[i] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    if (tid < kBlk) *reinterpret_cast<uint4*>(sAugK + (tid & 7) * 16 + (tid >> 3) * 256) = make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -584,20 +600,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
     if (warp == kProducerWarp) {
         if (E > 0) {   // the whole warp runs the loop (converged): lane 0 issues the copies, every lane writes its share of the slabs
             int issued = 0, issued_b = 0;
-            // zero every slab once (columns 3..15 stay zero), ones for the keys
-            for (int i = lane; i < (int)((C::kStages * 2 + 1) * C::kAugBytes / 16); i += 32)
-                reinterpret_cast<uint4*>(sAugQ)[i] = make_uint4(0u, 0u, 0u, 0u);
-            __syncwarp();
-            for (int r = lane; r < kBlk; r += 32)
-                *reinterpret_cast<uint4*>(sAugK + (r & 7) * 16 + (r >> 3) * 256) = make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u);
-            if (lane == 0) {
-                mbar_expect_tx(&bar.fixed_full, 2 * C::kTile);
-#pragma unroll
-                for (int pn = 0; pn < C::kPanels; ++pn) {
-                    tma_load_4d(sK + pn * kPanel, &maps.k[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
-                    tma_load_4d(sV + pn * kPanel, &maps.v[lvl], pn * 64, (int)j0, h, b, &bar.fixed_full);
-                }
-            }
             const float inv_scale = 1.f / p.scale_log2;
             int hq = h * p.kv_group, eq = 0;                // query head and tile-within-head of stage e
             // this lane's four queries of a tile: their biases and D_t, fetched one tile ahead of the stage they go into
@@ -665,9 +667,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             const uint32_t q_lo = desc_lo_kmajor(smem_u32(sQ)), g_lo = desc_lo_kmajor(smem_u32(sdO));
             const uint32_t qt_lo = desc_lo_mnmajor(smem_u32(sQ), kPanel), gt_lo = desc_lo_mnmajor(smem_u32(sdO), kPanel);
             const uint32_t augk_lo = desc_lo_flat(smem_u32(sAugK)), augq_lo = desc_lo_flat(smem_u32(sAugQ));
-            auto issue_s = [&](int e) -> bool {             // S^T(e) = K Q(e)^T   (P^T(e-1), which shares the columns, was consumed by dV(e-1) issued before)
+            auto issue_s = [&](int e) {                     // S^T(e) = K Q(e)^T   (P^T(e-1), which shares the columns, was consumed by dV(e-1) issued before; Q(e) has landed)
                 const int s = e % C::kStages;
-                if (!mbar_wait_warp(&bar.a_full[s], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
                 tc_fence_after();
                 const uint32_t qa = q_lo + s * (C::kTile >> 4);
 #pragma unroll
@@ -675,7 +676,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                     mma_ss_elect(tmem + kColS, make_desc(k_lo + kstep_off(k, kPanel)), make_desc(qa + kstep_off(k, kPanel)), C::kIdescS, k > 0);
                 mma_ss_elect(tmem + kColS, make_desc_flat(augk_lo), make_desc_flat(augq_lo + s * (2 * C::kAugBytes >> 4)), C::kIdescS, 1u);   // + bias_t / scale
                 mma_commit_elect(&bar.s_full[0]);
-                return true;
             };
             auto issue_dp = [&](int e) -> bool {            // dP^T(e) = V dO(e)^T
                 if (!mbar_wait_warp(&bar.b_full[e % C::kStages], (uint32_t)(e / C::kStages) & 1u, abortp)) return false;
@@ -688,7 +688,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                 mma_commit_elect(&bar.dp_full);
                 return true;
             };
-            if (ok) ok = issue_s(0);
+            if (ok) ok = mbar_wait_warp(&bar.a_full[0], 0, abortp);
+            if (ok) issue_s(0);
             if (ok) ok = issue_dp(0);
             for (int e = 0; e < E && ok; ++e) {
                 const int s = e % C::kStages;
@@ -708,16 +709,37 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
                 }
                 if (!ok) break;
                 mma_commit_elect(&bar.b_empty[s]);                     // dO(e) has had its last reader
-                if (e + 1 < E && !issue_s(e + 1)) { ok = false; break; }
+                // S^T(e+1) needs Q(e+1), which can only be requested once dK(e-1) has released its stage; dK(e) needs dS^T(e)
+                // from the element-wise threads.  Either may be ready first, and neither may wait for the other (a late
+                // dK delays the release, the release the copy, the copy the next S^T): poll both.
+                {
+                    const int sn = (e + 1) % C::kStages;
+                    const uint32_t phn = (uint32_t)((e + 1) / C::kStages) & 1u;
+                    bool s_out = e + 1 >= E;
+                    int dk_part = 0;
+                    const unsigned long long t0 = gtimer();
+                    while (!s_out || dk_part < 2) {
+                        bool moved = false;
+                        if (!s_out && __all_sync(0xffffffffu, mbar_try(&bar.a_full[sn], phn))) {
+                            issue_s(e + 1);
+                            s_out = moved = true;
+                        }
+                        if (dk_part < 2 && __all_sync(0xffffffffu, mbar_try(&bar.ds_part[dk_part], (uint32_t)e & 1u))) {
+                            tc_fence_after();
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
-                    if (!mbar_wait_warp(&bar.ds_part[part], (uint32_t)e & 1u, abortp)) { ok = false; break; }
-                    tc_fence_after();
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int k = (i >> 1) * 4 + part * 2 + (i & 1);
-                        mma_ts_elect(tmem + kColDK, tmem + kColDP + packed_half_col(k), make_desc(qta + k * (2048 >> 4)), C::kIdescAcc,
-                               (e > 0 || part > 0 || i > 0) ? 1u : 0u);
+                            for (int i = 0; i < 4; ++i) {
+                                const int k = (i >> 1) * 4 + dk_part * 2 + (i & 1);
+                                mma_ts_elect(tmem + kColDK, tmem + kColDP + packed_half_col(k), make_desc(qta + k * (2048 >> 4)), C::kIdescAcc,
+                                       (e > 0 || dk_part > 0 || i > 0) ? 1u : 0u);
+                            }
+                            ++dk_part;
+                            moved = true;
+                        }
+                        if (!moved) {                            // bounded like every other wait of the kernel
+                            bool give_up = abortp->abort != 0;
+                            if (!give_up && gtimer() - t0 > abortp->limit_ns) { abortp->abort = 1; give_up = true; }
+                            if (__any_sync(0xffffffffu, give_up)) { ok = false; break; }
+                        }
                     }
                 }
                 if (!ok) break;
