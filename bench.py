@@ -62,7 +62,7 @@ NCU_TRAFFIC = {
     "l2_summary_seg_kernel@s3": (101.000704e6 + 55.384064e6, 12288.0 / 32768.0, "l2_summary_seg_kernel_s3p.md", "summary_seg.cu", "6e2dcc00fbde"),   # 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8, "fuse_kv_kernel_f3p.md", "fuse_kv.cu", "3becacc721a4"),
     "decode_paged_kernel@g4": (293.682688e6 + 3.988480e6, 1 * 4, "decode_paged_kernel_g4p.md", "decode_paged.cu", "712e1e791061"),   # one of the four sequences (g4p)
-    "l3_index_kernel@r3": (134.308864e6 + 4.333824e6, 1, "l3_index_kernel_r3p.md", "l3.cu", "614940969b90"),            # one of the four sequences (r3p)
+    "l3_index_kernel@r3": (134.301696e6 + 3.607552e6, 1, "l3_index_kernel_r3p.md", "l3.cu", "6e05d1bc7821"),            # one of the four sequences (r3p)
 }
 
 

@@ -100,24 +100,30 @@ __global__ void __launch_bounds__(kIdxThreads, 4) l3_index_kernel(const L3IndexP
         const long long pair = base + lane;
         const float* sv = s + lane * pitch;
         for (int j0 = warp * kIdxBitsPerWarp; j0 < p.bits; j0 += (kIdxThreads / 32) * kIdxBitsPerWarp) {
-            float a[kIdxBitsPerWarp];
+            // two chains per instruction (fma.rn.f32x2: each half is the same correctly rounded fma as fmaf)
+            unsigned long long a2[kIdxBitsPerWarp / 2];
 #pragma unroll
-            for (int j = 0; j < kIdxBitsPerWarp; ++j) a[j] = 0.f;
+            for (int j = 0; j < kIdxBitsPerWarp / 2; ++j) a2[j] = 0ull;          // two +0.f
             const float* pj = projT + j0;
             for (int i = 0; i < DH; ++i) {
                 const float x = sv[i];
+                unsigned long long x2;
+                asm("mov.b64 %0, {%1, %1};" : "=l"(x2) : "f"(x));
 #pragma unroll
                 for (int v = 0; v < kIdxBitsPerWarp / 4; ++v) {
-                    const float4 pr = *reinterpret_cast<const float4*>(pj + (size_t)i * ppitch + 4 * v);
-                    a[4 * v] = fmaf(pr.x, x, a[4 * v]);
-                    a[4 * v + 1] = fmaf(pr.y, x, a[4 * v + 1]);
-                    a[4 * v + 2] = fmaf(pr.z, x, a[4 * v + 2]);
-                    a[4 * v + 3] = fmaf(pr.w, x, a[4 * v + 3]);
+                    const ulonglong2 pr = *reinterpret_cast<const ulonglong2*>(pj + (size_t)i * ppitch + 4 * v);   // bits 4v..4v+3 of column i
+                    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a2[2 * v]) : "l"(pr.x), "l"(x2));
+                    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a2[2 * v + 1]) : "l"(pr.y), "l"(x2));
                 }
             }
             unsigned half = 0u;
 #pragma unroll
-            for (int j = 0; j < kIdxBitsPerWarp; ++j) half |= (a[j] >= 0.f ? 1u : 0u) << j;
+            for (int j = 0; j < kIdxBitsPerWarp / 2; ++j) {
+                float lo, hi;
+                asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a2[j]));
+                half |= (lo >= 0.f ? 1u : 0u) << (2 * j);
+                half |= (hi >= 0.f ? 1u : 0u) << (2 * j + 1);
+            }
             // bits j0..j0+15 are one 16-bit half of word j0 / 32 (low half first)
             if (pair < pairs) codes16[(pair * words) * 2 + j0 / 16] = (unsigned short)half;
         }
