@@ -647,7 +647,7 @@ def oracle_sample(name, budget_rows=None):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "f3", "s3", "g4", "r3", "c3p", "c4p", "c5p", "f3p", "s3p", "g4p", "r3p"])
     ap.add_argument("--legs", default="c4,c5,c2,f3,s3,g4,r3", help="other configurations measured after the primary one ('' = none)")
