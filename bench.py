@@ -57,8 +57,8 @@ NCU_TRAFFIC = {
     "fwd_tc_kernel@c3": (376.523776e6 + 61.946368e6, 1 * 8, "fwd_tc_kernel_c3p.md", "fwd_tc.cu", "58f08d0c47e4"),
     "fwd_tc_kernel64@c2": (204.546304e6 + 28.208640e6, 8 * 16, "fwd_tc_kernel64_c2.md", "fwd_tc.cu", "58f08d0c47e4"),   # the whole configuration
     "decode_partial_kernel@c4": (1.476476e9 + 5.132288e6, 2 * 32, "decode_partial_kernel_c4p.md", "decode.cu", "ed9d09920f1b"),
-    "bwd_dq_tc_kernel@c5": (220.273920e6 + 27.224320e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "fe3660526f61"),
-    "bwd_dkv_tc_kernel@c5": (220.317184e6 + 114.672128e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "fe3660526f61"),
+    "bwd_dq_tc_kernel@c5": (220.275200e6 + 27.056128e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "5b543af267de"),
+    "bwd_dkv_tc_kernel@c5": (220.271872e6 + 114.367232e6, 1 * 16, "bwd_tc_kernels_c5p.md", "bwd_tc.cu", "5b543af267de"),
     "l2_summary_seg_kernel@s3": (101.000704e6 + 55.384064e6, 12288.0 / 32768.0, "l2_summary_seg_kernel_s3p.md", "summary_seg.cu", "6e2dcc00fbde"),   # 12288 of the 32768 tokens
     "fuse_kv_kernel@f3": (403.137024e6 + 83.414784e6, 1 * 8, "fuse_kv_kernel_f3p.md", "fuse_kv.cu", "3becacc721a4"),
     "decode_paged_kernel@g4": (293.682688e6 + 3.988480e6, 1 * 4, "decode_paged_kernel_g4p.md", "decode_paged.cu", "712e1e791061"),   # one of the four sequences (g4p)

@@ -66,8 +66,11 @@ typedef enum { MKA_ROUTE_SOFT = 0, MKA_ROUTE_UNIFORM = 1, MKA_ROUTE_TOP1 = 2, MK
 #define MKA_FLAG_TEST_STALL 0x80000000u /* test hook of mka_fwd (tensor-core kernel, dense levels): the loader of every
                                            CTA leaves out its last key tile, so the wait for that tile runs into the
                                            limit of mka_set_wait_limit_us and the call ends with MKA_ERR_TIMEOUT in
-                                           the status word; O and LSE of such a call are invalid.  Exists so that
-                                           the give-up path can be exercised without a fault or a hang. */
+                                           the status word; O and LSE of such a call are invalid.  In mka_bwd
+                                           (tensor-core kernels) the loader of every CTA of the dK/dV kernel leaves
+                                           out its last query tile, with the same end; the gradients of such a call
+                                           are invalid.  Exists so that the give-up path can be exercised without a
+                                           fault or a hang. */
 
 /* which = argument of mka_workspace_bytes */
 #define MKA_WS_FWD 0

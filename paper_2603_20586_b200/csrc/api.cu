@@ -500,6 +500,7 @@ mka_status mka_bwd(const mka_shape* s, const void* Q, const mka_level L[3], cons
     p.stats = reinterpret_cast<float*>(w);
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d;
     p.window = s->window; p.q_offset = s->q_offset; p.scale = resolve_scale(s); p.kv_group = kv_group_of(s);
+    p.test_stall = (s->flags & MKA_FLAG_TEST_STALL) ? 1 : 0;
     const bool tc = !(s->flags & MKA_FLAG_FORCE_SIMT) && bwd_tc_eligible(p, s->dtype);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 16, cs) != cudaSuccess) return MKA_ERR_CUDA;

@@ -66,6 +66,7 @@ struct BwdTcParams {
     int kv_tiles[3];          // 128-row key tiles per level
     unsigned int* status;
     unsigned long long wait_limit_ns;
+    int test_stall;           // test hook: the dK/dV kernel's loader leaves out the last query tile of every CTA
 };
 
 // v as a sum of three bf16 terms (exact to 2^-25 |v|) in the first three of eight bf16 slots of a 16-byte core-matrix row;
@@ -615,6 +616,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_dkv_tc_kernel(const __grid_co
             for (int e = 0; e < E; ++e) {
                 const int s = e % C::kStages;
                 const uint32_t ph = (uint32_t)(e / C::kStages) & 1u;
+                if (p.test_stall && e == E - 1) break;                 // test hook: the last tile never arrives
                 const int tt = (first + eq) * kBlk;
                 const float bv[4] = {bq.x, bq.y, bq.z, bq.w}, dv[4] = {dq.x, dq.y, dq.z, dq.w};
                 if (!mbar_wait_warp(&bar.b_empty[s], ph ^ 1u, abortp)) break;
@@ -910,6 +912,7 @@ cudaError_t launch_t(const BwdParams& bp, unsigned int* status_word, cudaStream_
     p.scale = bp.scale; p.scale_log2 = bp.scale * kLog2e;
     p.status = status_word;
     p.wait_limit_ns = wait_limit_ns();
+    p.test_stall = bp.test_stall;
 
     // both kernels move 128-row tiles (box = 64 columns x 128 rows)
     {

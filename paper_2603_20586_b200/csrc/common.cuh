@@ -150,6 +150,7 @@ struct BwdParams {
     int window, q_offset;
     float scale;
     int kv_group;     // query heads per KV head (>= 1); > 1 only on the tensor-core path
+    int test_stall;   // MKA_FLAG_TEST_STALL (tensor-core path): the dK/dV kernel's loader leaves out its last query tile
 };
 cudaError_t launch_bwd_simt(const BwdParams& p, int dtype, cudaStream_t st);
 cudaError_t launch_router_bwd(const void* R, int r_dtype, const float* dG, long long rows, int D, float* dW_r,
